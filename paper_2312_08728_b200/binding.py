@@ -1,0 +1,236 @@
+"""ctypes binding of the BMGD C ABI (include/bmgd.h).
+
+Argument marshalling only: every step of the computation runs in the CUDA library.
+torch is used for device memory (the workspace), pinned host memory and streams.
+There is no CPU fallback: if the library cannot be loaded, or no CUDA device is
+present, creating a handle raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import numpy as np
+import torch
+
+from . import build as _build
+from .inputs import DTYPE_BF16, DTYPE_F32, DTYPE_F64, LOSS_LINEAR, LOSS_LOGISTIC, LOSS_SOFTMAX
+
+BMGD_OK = 0
+ERR_ARG, ERR_ALLOC, ERR_CUDA, ERR_CAPACITY, ERR_TIMEOUT = -1, -2, -3, -4, -5
+ERR_NONFINITE, ERR_LAUNCH, ERR_UNIMPLEMENTED, ERR_STATE = -6, -7, -8, -9
+
+FLAG_FIXED_PARTITION = 1
+FLAG_NO_SLOTS = 2
+FLAG_TIMING = 4
+
+# every symbol include/bmgd.h declares
+EXPORTS = (
+    "bmgd_config_init", "bmgd_workspace_bytes", "bmgd_create", "bmgd_create_ex", "bmgd_destroy",
+    "bmgd_load_buffer", "bmgd_run_rounds", "bmgd_run_rounds_resident", "bmgd_sync", "bmgd_get_theta",
+    "bmgd_set_theta", "bmgd_get_stats", "bmgd_debug_perm", "bmgd_strerror", "bmgd_last_cuda_error",
+    "bmgd_version",
+)
+
+
+class BmgdConfig(ctypes.Structure):
+    _fields_ = [
+        ("N", ctypes.c_int64), ("p", ctypes.c_int32), ("K", ctypes.c_int32), ("loss", ctypes.c_int32),
+        ("dtype", ctypes.c_int32), ("C", ctypes.c_int32), ("Rc", ctypes.c_int32), ("device", ctypes.c_int32),
+        ("flags", ctypes.c_uint32), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_int64),
+        ("compute_stream", ctypes.c_void_p), ("timeout_ms", ctypes.c_double),
+        ("cluster_size", ctypes.c_int32), ("ctas_per_chain", ctypes.c_int32),
+        ("threads_per_cta", ctypes.c_int32), ("pipeline_depth", ctypes.c_int32),
+        ("reserved", ctypes.c_int32 * 8),
+    ]
+
+
+class BmgdStats(ctypes.Structure):
+    _fields_ = [
+        ("launches", ctypes.c_int64), ("steps", ctypes.c_int64), ("sample_grads", ctypes.c_int64),
+        ("h2d_bytes", ctypes.c_int64), ("kernel_ms", ctypes.c_double), ("h2d_ms", ctypes.c_double),
+        ("grid_ctas", ctypes.c_int32), ("cluster_size", ctypes.c_int32), ("ctas_per_chain", ctypes.c_int32),
+        ("threads_per_cta", ctypes.c_int32), ("pipeline_depth", ctypes.c_int32), ("smem_bytes", ctypes.c_int32),
+        ("chains_in_flight", ctypes.c_int32), ("reserved", ctypes.c_int32),
+    ]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_ if k != "reserved"}
+
+
+class BmgdError(RuntimeError):
+    def __init__(self, status: int, where: str, cuda: int = 0):
+        self.status = status
+        self.cuda_error = cuda
+        msg = load_library().bmgd_strerror(status).decode()
+        super().__init__(f"{where}: {msg} (status {status}" + (f", cudaError {cuda})" if cuda else ")"))
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def load_library(path: Optional[str] = None) -> ctypes.CDLL:
+    """Load libbmgd.so (building it first if its sources are newer) and declare the ABI."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    if path is None:
+        path = _build.LIB_PATH
+        if _build.is_stale():
+            if _build.find_nvcc() is not None:
+                _build.build()
+            elif not os.path.exists(path):
+                raise RuntimeError("libbmgd.so is not built and nvcc is not available")
+    L = ctypes.CDLL(path)
+    vp, i32, i64, u32, u64, dbl = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint32,
+                                  ctypes.c_uint64, ctypes.c_double)
+    P = ctypes.POINTER
+    L.bmgd_config_init.argtypes = [P(BmgdConfig)]; L.bmgd_config_init.restype = None
+    L.bmgd_workspace_bytes.argtypes = [P(BmgdConfig), P(i64)]
+    L.bmgd_create.argtypes = [i64, i32, i32, i32, P(vp)]
+    L.bmgd_create_ex.argtypes = [P(BmgdConfig), P(vp)]
+    L.bmgd_destroy.argtypes = [vp]
+    L.bmgd_load_buffer.argtypes = [vp, vp, vp, i64, vp, P(i32)]
+    L.bmgd_run_rounds.argtypes = [vp, i32, i32, i32, dbl, u64]
+    L.bmgd_run_rounds_resident.argtypes = [vp, vp, vp, i64, i32, i32, dbl, u64]
+    L.bmgd_sync.argtypes = [vp]
+    L.bmgd_get_theta.argtypes = [vp, vp, i64]
+    L.bmgd_set_theta.argtypes = [vp, vp, i64]
+    L.bmgd_get_stats.argtypes = [vp, P(BmgdStats)]
+    L.bmgd_debug_perm.argtypes = [vp, u64, u32, u32, u32, vp]
+    L.bmgd_strerror.argtypes = [ctypes.c_int]; L.bmgd_strerror.restype = ctypes.c_char_p
+    L.bmgd_last_cuda_error.argtypes = [vp]
+    L.bmgd_version.argtypes = []
+    for name in EXPORTS:
+        if getattr(L, name).restype is None or name in ("bmgd_strerror",):
+            continue
+        getattr(L, name).restype = ctypes.c_int
+    if path == _build.LIB_PATH:
+        _lib = L
+    return L
+
+
+_NP_THETA = {DTYPE_F64: np.float64, DTYPE_F32: np.float32, DTYPE_BF16: np.float32}
+
+
+class Bmgd:
+    """One BMGD handle: theta for Rc chains, two device buffer slots, a compute stream.
+
+    Mirrors the C calls one to one: load_buffer, run_rounds, run_rounds_resident, sync,
+    get_theta, set_theta, get_stats, debug_perm.
+    """
+
+    def __init__(self, N: int, p: int, K: int, loss: int = LOSS_LINEAR, dtype: int = DTYPE_F32, C: int = 1,
+                 Rc: int = 1, device: int = 0, flags: int = 0, cluster_size: int = 0, ctas_per_chain: int = 0,
+                 threads_per_cta: int = 0, pipeline_depth: int = 0, timeout_ms: float = 0.0,
+                 use_torch_stream: bool = False):
+        if not torch.cuda.is_available():
+            raise RuntimeError("BMGD needs a CUDA device; there is no CPU path")
+        self._lib = load_library()
+        self._h = ctypes.c_void_p()
+        cfg = BmgdConfig()
+        self._lib.bmgd_config_init(ctypes.byref(cfg))
+        cfg.N, cfg.p, cfg.K, cfg.loss, cfg.dtype, cfg.C, cfg.Rc = N, p, K, loss, dtype, C, Rc
+        cfg.device, cfg.flags = device, flags
+        cfg.cluster_size, cfg.ctas_per_chain = cluster_size, ctas_per_chain
+        cfg.threads_per_cta, cfg.pipeline_depth, cfg.timeout_ms = threads_per_cta, pipeline_depth, timeout_ms
+        need = ctypes.c_int64()
+        self._check(self._lib.bmgd_workspace_bytes(ctypes.byref(cfg), ctypes.byref(need)), "bmgd_workspace_bytes")
+        self.device = torch.device("cuda", device)
+        # device memory comes from torch's allocator; the library carves it up
+        self._workspace = torch.empty(need.value + 256, dtype=torch.uint8, device=self.device)
+        base = (self._workspace.data_ptr() + 255) // 256 * 256
+        cfg.workspace, cfg.workspace_bytes = base, need.value
+        if use_torch_stream:
+            self._stream = torch.cuda.current_stream(self.device)
+            cfg.compute_stream = self._stream.cuda_stream
+        self.cfg = cfg
+        self.N, self.p, self.K, self.loss, self.dtype, self.C, self.Rc = N, p, K, loss, dtype, C, Rc
+        self._check(self._lib.bmgd_create_ex(ctypes.byref(cfg), ctypes.byref(self._h)), "bmgd_create_ex")
+        self._keep = []  # host tensors whose copies may still be in flight
+
+    # -- helpers
+    def _check(self, status: int, where: str, allow=()):
+        if status != BMGD_OK and status not in allow:
+            cuda = self._lib.bmgd_last_cuda_error(self._h) if self._h else 0
+            raise BmgdError(status, where, cuda)
+        return status
+
+    @property
+    def theta_shape(self) -> Tuple[int, ...]:
+        return (self.Rc, self.p, self.C) if self.loss == LOSS_SOFTMAX else (self.Rc, self.p)
+
+    # -- the calls
+    def load_buffer(self, host_x: torch.Tensor, host_y: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> int:
+        """Start the host-to-device copy of one buffer; returns the slot id."""
+        if host_x.device.type != "cpu" or host_y.device.type != "cpu":
+            raise ValueError("load_buffer takes host tensors")
+        if not (host_x.is_contiguous() and host_y.is_contiguous()):
+            raise ValueError("host buffers must be contiguous")
+        rows = host_x.shape[0]
+        slot = ctypes.c_int32(-1)
+        s = stream.cuda_stream if stream is not None else None
+        self._check(self._lib.bmgd_load_buffer(self._h, host_x.data_ptr(), host_y.data_ptr(), rows, s,
+                                               ctypes.byref(slot)), "bmgd_load_buffer")
+        self._keep.append((host_x, host_y))
+        if len(self._keep) > 4:
+            self._keep.pop(0)
+        return slot.value
+
+    def run_rounds(self, slot: int, rounds: int, batch_size: int, lr: float, seed: int) -> None:
+        self._check(self._lib.bmgd_run_rounds(self._h, slot, rounds, batch_size, float(lr),
+                                              int(seed) & 0xFFFFFFFFFFFFFFFF), "bmgd_run_rounds")
+
+    def run_rounds_resident(self, dev_x: torch.Tensor, dev_y: torch.Tensor, rounds: int, batch_size: int,
+                            lr: float, seed: int) -> None:
+        if dev_x.device != self.device or dev_y.device != self.device:
+            raise ValueError("resident buffers must live on the handle's device")
+        if not (dev_x.is_contiguous() and dev_y.is_contiguous()):
+            raise ValueError("resident buffers must be contiguous")
+        self._check(self._lib.bmgd_run_rounds_resident(self._h, dev_x.data_ptr(), dev_y.data_ptr(), dev_x.shape[0],
+                                                       rounds, batch_size, float(lr),
+                                                       int(seed) & 0xFFFFFFFFFFFFFFFF), "bmgd_run_rounds_resident")
+
+    def sync(self) -> None:
+        self._check(self._lib.bmgd_sync(self._h), "bmgd_sync")
+        self._keep.clear()
+
+    def get_theta(self, allow_nonfinite: bool = False) -> np.ndarray:
+        out = np.empty(self.theta_shape, dtype=_NP_THETA[self.dtype])
+        self._check(self._lib.bmgd_get_theta(self._h, out.ctypes.data, out.nbytes), "bmgd_get_theta",
+                    allow=(ERR_NONFINITE,) if allow_nonfinite else ())
+        return out
+
+    def set_theta(self, theta: np.ndarray) -> None:
+        a = np.ascontiguousarray(theta, dtype=_NP_THETA[self.dtype]).reshape(self.theta_shape)
+        self._check(self._lib.bmgd_set_theta(self._h, a.ctypes.data, a.nbytes), "bmgd_set_theta")
+
+    def get_stats(self) -> dict:
+        st = BmgdStats()
+        self._check(self._lib.bmgd_get_stats(self._h, ctypes.byref(st)), "bmgd_get_stats")
+        return st.as_dict()
+
+    def debug_perm(self, seed: int, chain: int, rnd: int, N0: int) -> np.ndarray:
+        out = np.empty(N0, dtype=np.uint32)
+        self._check(self._lib.bmgd_debug_perm(self._h, int(seed) & 0xFFFFFFFFFFFFFFFF, chain, rnd, N0,
+                                              out.ctypes.data), "bmgd_debug_perm")
+        return out
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h:
+            self._lib.bmgd_destroy(self._h)
+            self._h = ctypes.c_void_p()
+        self._workspace = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()

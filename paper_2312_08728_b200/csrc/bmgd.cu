@@ -1,0 +1,694 @@
+// Host side of the BMGD library: the C ABI of include/bmgd.h, the handle, the two buffer slots
+// with their copy/compute event ordering (the buffering step of Section 2.1 overlapped with the
+// computation step), launch-shape selection and kernel dispatch.
+#include "../../include/bmgd.h"
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "glm_kernel.cuh"
+#include "softmax_kernel.cuh"
+
+namespace {
+
+using bmgdk::GlmParams;
+
+constexpr int64_t kAlign = 256;
+constexpr int kMaxClustersForExchange = 160;  // upper bound on clusters in one grid (148 SMs)
+constexpr int kVersion = 1000;
+
+inline int64_t align_up(int64_t v, int64_t a = kAlign) { return (v + a - 1) / a * a; }
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+struct EventPair {
+    cudaEvent_t a, b;
+};
+
+struct Layout {
+    int64_t slot_x[2], slot_y[2];
+    int64_t theta, ll, status, softmax_scratch;
+    int64_t total;
+};
+
+}  // namespace
+
+struct bmgd {
+    bmgd_config cfg;
+    int device = 0;
+    int sm_count = 0;
+    int smem_optin = 0;
+    int64_t N0cap = 0;
+    int xb = 4, yb = 4, tb = 4;  // bytes per stored x, y, theta element
+    int num_slots = 2;
+    unsigned char* base = nullptr;
+    bool owns_base = false;
+    Layout lay{};
+    cudaStream_t compute = nullptr;
+    bool owns_stream = false;
+    cudaEvent_t loaded[2] = {nullptr, nullptr};
+    cudaEvent_t freed[2] = {nullptr, nullptr};
+    int64_t slot_rows[2] = {0, 0};
+    bool slot_has_data[2] = {false, false};
+    int next_slot = 0;
+    uint64_t tag_base = 0;
+    int last_cuda = 0;
+    bmgd_stats stats{};
+    std::vector<EventPair> kernel_events, copy_events, event_pool;
+    uint64_t timeout_ns = 2000000000ull;
+};
+
+namespace {
+
+int cuda_fail(bmgd* h, cudaError_t e) {
+    if (h) h->last_cuda = (int)e;
+    cudaGetLastError();  // clear the sticky-less error state
+    return BMGD_ERR_CUDA;
+}
+
+#define BMGD_CUDA(h, call)                                   \
+    do {                                                     \
+        cudaError_t e__ = (call);                            \
+        if (e__ != cudaSuccess) return cuda_fail((h), e__);  \
+    } while (0)
+
+int elem_bytes_x(int dtype) { return dtype == BMGD_F64 ? 8 : dtype == BMGD_F32 ? 4 : 2; }
+int elem_bytes_theta(int dtype) { return dtype == BMGD_F64 ? 8 : 4; }
+
+int validate(const bmgd_config* c) {
+    if (!c) return BMGD_ERR_ARG;
+    if (c->N <= 0 || c->p <= 0 || c->K <= 0 || c->K > c->N) return BMGD_ERR_ARG;
+    if (c->loss < BMGD_LOSS_LINEAR || c->loss > BMGD_LOSS_SOFTMAX) return BMGD_ERR_ARG;
+    if (c->dtype < BMGD_F64 || c->dtype > BMGD_BF16X_F32W) return BMGD_ERR_ARG;
+    if (c->Rc < 1 || c->Rc > 65536) return BMGD_ERR_ARG;
+    if (c->loss == BMGD_LOSS_SOFTMAX) {
+        if (c->C < 2 || c->C > 16) return c->C < 2 ? BMGD_ERR_ARG : BMGD_ERR_UNIMPLEMENTED;
+        if (c->dtype != BMGD_BF16X_F32W) return BMGD_ERR_UNIMPLEMENTED;
+        if (c->Rc != 1) return BMGD_ERR_UNIMPLEMENTED;
+    } else {
+        if (c->C != 1) return BMGD_ERR_ARG;
+        if (c->dtype == BMGD_BF16X_F32W) return BMGD_ERR_UNIMPLEMENTED;
+    }
+    const int64_t N0 = (c->N + c->K - 1) / c->K;
+    if (N0 > 0x7FFFFFFFll) return BMGD_ERR_ARG;
+    for (int i = 0; i < 8; ++i)
+        if (c->reserved[i] != 0) return BMGD_ERR_ARG;
+    if (c->cluster_size != 0 && c->cluster_size != 1 && c->cluster_size != 2 && c->cluster_size != 4 &&
+        c->cluster_size != 8 && c->cluster_size != 16)
+        return BMGD_ERR_ARG;
+    if (c->threads_per_cta != 0 && (c->threads_per_cta % 32 != 0 || c->threads_per_cta < 256 || c->threads_per_cta > 1024))
+        return BMGD_ERR_ARG;
+    if (c->pipeline_depth != 0 && (c->pipeline_depth < 2 || c->pipeline_depth > 16)) return BMGD_ERR_ARG;
+    if (c->ctas_per_chain < 0) return BMGD_ERR_ARG;
+    if (c->workspace && ((uintptr_t)c->workspace % kAlign) != 0) return BMGD_ERR_ARG;
+    return BMGD_OK;
+}
+
+Layout make_layout(const bmgd_config* c) {
+    Layout L{};
+    const int64_t N0 = (c->N + c->K - 1) / c->K;
+    const int xb = elem_bytes_x(c->dtype), tb = elem_bytes_theta(c->dtype);
+    const int yb = c->loss == BMGD_LOSS_SOFTMAX ? 4 : tb;
+    int64_t off = 0;
+    const int slots = (c->flags & BMGD_FLAG_NO_SLOTS) ? 0 : 2;
+    for (int s = 0; s < 2; ++s) {
+        L.slot_x[s] = off; if (s < slots) off += align_up(N0 * c->p * xb);
+        L.slot_y[s] = off; if (s < slots) off += align_up(N0 * yb);
+    }
+    L.theta = off; off += align_up((int64_t)c->Rc * c->p * c->C * tb);
+    L.ll = off;
+    if (c->loss != BMGD_LOSS_SOFTMAX) off += align_up((int64_t)2 * kMaxClustersForExchange * c->p * 2 * 8);
+    L.status = off; off += kAlign;
+    L.softmax_scratch = off;
+    if (c->loss == BMGD_LOSS_SOFTMAX) off += align_up(bmgdk::softmax_scratch_bytes(c->p, c->C));
+    L.total = off;
+    return L;
+}
+
+// ------------------------------------------------------------------ GLM kernel table
+
+typedef void (*GlmKernel)(const GlmParams);
+
+struct GlmVariant {
+    GlmKernel fn;
+    int vec, lpr, kch, maxt;
+    int cap() const { return vec * lpr * kch; }
+    int max_threads() const { return maxt; }
+};
+
+template <typename T>
+const GlmVariant* glm_variants(bool aligned16, int* count) {
+    constexpr int V = 16 / (int)sizeof(T);
+    static const GlmVariant wide[] = {
+        {bmgdk::glm_kernel<T, V, 8, 1>, V, 8, 1, bmgdk::glm_max_threads<T, V, 1>()},  {bmgdk::glm_kernel<T, V, 8, 2>, V, 8, 2, bmgdk::glm_max_threads<T, V, 2>()},
+        {bmgdk::glm_kernel<T, V, 8, 4>, V, 8, 4, bmgdk::glm_max_threads<T, V, 4>()},  {bmgdk::glm_kernel<T, V, 8, 8>, V, 8, 8, bmgdk::glm_max_threads<T, V, 8>()},
+        {bmgdk::glm_kernel<T, V, 16, 8>, V, 16, 8, bmgdk::glm_max_threads<T, V, 8>()}, {bmgdk::glm_kernel<T, V, 32, 8>, V, 32, 8, bmgdk::glm_max_threads<T, V, 8>()},
+    };
+    static const GlmVariant narrow[] = {
+        {bmgdk::glm_kernel<T, 1, 32, 1>, 1, 32, 1, bmgdk::glm_max_threads<T, 1, 1>()}, {bmgdk::glm_kernel<T, 1, 32, 2>, 1, 32, 2, bmgdk::glm_max_threads<T, 1, 2>()},
+        {bmgdk::glm_kernel<T, 1, 32, 4>, 1, 32, 4, bmgdk::glm_max_threads<T, 1, 4>()}, {bmgdk::glm_kernel<T, 1, 32, 8>, 1, 32, 8, bmgdk::glm_max_threads<T, 1, 8>()},
+    };
+    if (aligned16) { *count = 6; return wide; }
+    *count = 4;
+    return narrow;
+}
+
+const GlmVariant* pick_variant(int dtype, int p, bool aligned16) {
+    int cnt = 0;
+    const GlmVariant* v = dtype == BMGD_F64 ? glm_variants<double>(aligned16, &cnt) : glm_variants<float>(aligned16, &cnt);
+    for (int i = 0; i < cnt; ++i)
+        if (v[i].cap() >= p) return &v[i];
+    return nullptr;
+}
+
+int floor_pow2(int v) {
+    int r = 1;
+    while (r * 2 <= v) r *= 2;
+    return r;
+}
+
+struct LaunchShape {
+    int S, cpc, nteams, threads, depth, passes, pitch, smem;
+};
+
+int max_active_clusters(bmgd* h, GlmKernel fn, int S, int threads, int smem, int* out) {
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3((unsigned)(S * h->sm_count), 1, 1);
+    lc.blockDim = dim3((unsigned)threads, 1, 1);
+    lc.dynamicSmemBytes = (size_t)smem;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)S; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    lc.attrs = at; lc.numAttrs = 1;
+    int n = 0;
+    BMGD_CUDA(h, cudaOccupancyMaxActiveClusters(&n, (const void*)fn, &lc));
+    *out = n;
+    return BMGD_OK;
+}
+
+int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* out) {
+    const bmgd_config& c = h->cfg;
+    const int eb = h->tb;
+    const int gpw = 32 / var->lpr;
+    const int pcap = var->cap();
+    LaunchShape L{};
+    L.threads = c.threads_per_cta ? std::min(c.threads_per_cta, var->max_threads())
+                                  : ((c.Rc > 1 && var->max_threads() >= 512) ? 512 : 256);
+    const int warps = L.threads / 32;
+    const int spp = warps * gpw;
+    L.pitch = (int)align_up((int64_t)c.p * eb, 16);
+
+    // cluster size
+    int S = c.cluster_size;
+    if (S == 0) {
+        if (c.Rc > 1) S = std::min(8, floor_pow2(std::max(1, h->sm_count / c.Rc)));
+        else S = 8;
+        // do not spread a mini-batch thinner than 8 rows per CTA
+        while (S > 1 && n / S < 8) S /= 2;
+    }
+    L.S = S;
+
+    // fixed shared memory and a first guess at the depth, to ask the occupancy calculator
+    auto smem_for = [&](int depth) {
+        return bmgdk::glm_smem_plan(warps, gpw, depth, L.pitch, pcap, eb, S).total_bytes;
+    };
+    const int stage_bytes = spp * (L.pitch + 16);
+    int depth = c.pipeline_depth ? c.pipeline_depth : (int)std::min<int64_t>(16, std::max<int64_t>(3, (128 * 1024) / stage_bytes));
+    while (depth > 2 && smem_for(depth) > h->smem_optin) --depth;
+    if (smem_for(depth) > h->smem_optin) return BMGD_ERR_UNIMPLEMENTED;
+    L.depth = depth;
+    L.smem = smem_for(depth);
+
+    BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn, cudaFuncAttributeMaxDynamicSharedMemorySize, L.smem));
+    if (S > 8) BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+    int max_clusters = h->sm_count;
+    if (S > 1) {
+        int rc = max_active_clusters(h, var->fn, S, L.threads, L.smem, &max_clusters);
+        if (rc != BMGD_OK) return rc;
+    }
+    if (max_clusters < 1) return BMGD_ERR_LAUNCH;
+    max_clusters = std::min(max_clusters, kMaxClustersForExchange);
+
+    if (c.Rc > 1 && c.ctas_per_chain == 0) {
+        L.cpc = 1;
+        L.nteams = std::min(c.Rc, max_clusters);
+    } else {
+        int cpc;
+        if (c.ctas_per_chain) {
+            if (c.ctas_per_chain % S != 0) return BMGD_ERR_ARG;
+            cpc = c.ctas_per_chain / S;
+        } else {
+            cpc = std::max(1, std::min(max_clusters, n / (8 * S)));
+        }
+        cpc = std::min(cpc, bmgdk::kMaxCpc);
+        if (cpc > max_clusters) return BMGD_ERR_LAUNCH;
+        L.cpc = cpc;
+        L.nteams = std::max(1, std::min(c.Rc, max_clusters / cpc));
+    }
+    const int G = L.cpc * S;
+    const int rows_per_cta = (n + G - 1) / G;
+    L.passes = std::max(1, (rows_per_cta + spp - 1) / spp);
+    (void)rows;
+    *out = L;
+    return BMGD_OK;
+}
+
+
+int take_events(bmgd* h, EventPair* ep) {
+    if (!h->event_pool.empty()) {
+        *ep = h->event_pool.back();
+        h->event_pool.pop_back();
+        return BMGD_OK;
+    }
+    BMGD_CUDA(h, cudaEventCreate(&ep->a));
+    BMGD_CUDA(h, cudaEventCreate(&ep->b));
+    return BMGD_OK;
+}
+
+int drain_events(bmgd* h, std::vector<EventPair>& v, double* acc) {
+    for (EventPair& ep : v) {
+        float ms = 0.f;
+        BMGD_CUDA(h, cudaEventSynchronize(ep.b));
+        BMGD_CUDA(h, cudaEventElapsedTime(&ms, ep.a, ep.b));
+        *acc += ms;
+        h->event_pool.push_back(ep);
+    }
+    v.clear();
+    return BMGD_OK;
+}
+
+int check_status_word(bmgd* h) {
+    int st[2] = {0, 0};
+    BMGD_CUDA(h, cudaMemcpy(st, h->base + h->lay.status, sizeof st, cudaMemcpyDeviceToHost));
+    if (st[0] != 0 || st[1] != 0) {
+        // report once, then clear so that the handle stays usable
+        cudaMemset(h->base + h->lay.status, 0, kAlign);
+        return st[0] != 0 ? st[0] : BMGD_ERR_TIMEOUT;
+    }
+    return BMGD_OK;
+}
+
+int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, int n, double lr, uint64_t seed) {
+    const bmgd_config& c = h->cfg;
+    const bool aligned16 = ((int64_t)c.p * h->tb) % 16 == 0 && ((uintptr_t)dx % 16) == 0;
+    const GlmVariant* var = pick_variant(c.dtype, c.p, aligned16);
+    if (!var) return BMGD_ERR_UNIMPLEMENTED;
+    if (((uintptr_t)dx % h->tb) != 0 || ((uintptr_t)dy % h->tb) != 0) return BMGD_ERR_ARG;
+    LaunchShape L{};
+    int rc = plan_glm(h, var, rows, n, &L);
+    if (rc != BMGD_OK) return rc;
+
+    const uint32_t M = (uint32_t)((rows + n - 1) / n);
+    const int chains_per_team = (c.Rc + L.nteams - 1) / L.nteams;
+    const uint64_t steps_per_team = (uint64_t)chains_per_team * (uint64_t)rounds * M;
+    if (steps_per_team >= 0xFFFFFFF0ull) return BMGD_ERR_ARG;
+    if (h->tag_base + steps_per_team >= 0xFFFFFFF0ull) {
+        // tags would wrap: wipe the packet area (on-stream, after earlier launches) and start over
+        BMGD_CUDA(h, cudaMemsetAsync(h->base + h->lay.ll, 0, (size_t)(h->lay.status - h->lay.ll), h->compute));
+        h->tag_base = 0;
+    }
+
+    GlmParams P{};
+    P.X = dx; P.y = dy;
+    P.theta = h->base + h->lay.theta;
+    P.ll = reinterpret_cast<unsigned long long*>(h->base + h->lay.ll);
+    P.status = reinterpret_cast<int*>(h->base + h->lay.status);
+    P.seed = seed;
+    P.timeout_ns = h->timeout_ns;
+    P.alpha = lr;
+    P.N0 = (uint32_t)rows; P.n = (uint32_t)n; P.M = M; P.T = rounds; P.p = c.p;
+    P.loss = c.loss; P.Rc = c.Rc; P.S = L.S; P.cpc = L.cpc; P.nteams = L.nteams;
+    P.passes = L.passes; P.depth = L.depth; P.pitch = L.pitch;
+    P.ll_stride = c.p * 2;
+    P.tag_base = (uint32_t)h->tag_base;
+    P.fixed_partition = (c.flags & BMGD_FLAG_FIXED_PARTITION) ? 1 : 0;
+    if ((int64_t)L.nteams * L.cpc > kMaxClustersForExchange) return BMGD_ERR_LAUNCH;
+
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3((unsigned)(L.nteams * L.cpc * L.S), 1, 1);
+    lc.blockDim = dim3((unsigned)L.threads, 1, 1);
+    lc.dynamicSmemBytes = (size_t)L.smem;
+    lc.stream = h->compute;
+    cudaLaunchAttribute at[2];
+    int na = 0;
+    if (L.S > 1) {
+        at[na].id = cudaLaunchAttributeClusterDimension;
+        at[na].val.clusterDim.x = (unsigned)L.S; at[na].val.clusterDim.y = 1; at[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    if (L.cpc > 1) {  // CTAs of different clusters wait on one another: they must all be resident
+        at[na].id = cudaLaunchAttributeCooperative;
+        at[na].val.cooperative = 1;
+        ++na;
+    }
+    lc.attrs = at; lc.numAttrs = (unsigned)na;
+
+    EventPair ep{};
+    const bool timing = (c.flags & BMGD_FLAG_TIMING) != 0;
+    if (timing) {
+        rc = take_events(h, &ep);
+        if (rc != BMGD_OK) return rc;
+        BMGD_CUDA(h, cudaEventRecord(ep.a, h->compute));
+    }
+    cudaError_t e = cudaLaunchKernelEx(&lc, var->fn, P);
+    if (e != cudaSuccess) {
+        h->last_cuda = (int)e;
+        cudaGetLastError();
+        if (timing) h->event_pool.push_back(ep);
+        return (e == cudaErrorCooperativeLaunchTooLarge || e == cudaErrorLaunchOutOfResources) ? BMGD_ERR_LAUNCH
+                                                                                                : BMGD_ERR_CUDA;
+    }
+    if (timing) {
+        BMGD_CUDA(h, cudaEventRecord(ep.b, h->compute));
+        h->kernel_events.push_back(ep);
+    }
+    h->tag_base += steps_per_team;
+    h->stats.launches += 1;
+    h->stats.steps += (int64_t)c.Rc * rounds * M;
+    h->stats.sample_grads += (int64_t)c.Rc * rounds * rows;
+    h->stats.grid_ctas = L.nteams * L.cpc * L.S;
+    h->stats.cluster_size = L.S;
+    h->stats.ctas_per_chain = L.cpc * L.S;
+    h->stats.threads_per_cta = L.threads;
+    h->stats.pipeline_depth = L.depth;
+    h->stats.smem_bytes = L.smem;
+    h->stats.chains_in_flight = L.nteams;
+    return BMGD_OK;
+}
+
+int run_any(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, int n, double lr, uint64_t seed) {
+    if (rows <= 0 || rows > 0x7FFFFFFFll || rounds < 0 || n <= 0 || !std::isfinite(lr)) return BMGD_ERR_ARG;
+    if (rounds == 0) return BMGD_OK;
+    if (n > rows) n = (int)rows;
+    if (h->cfg.loss == BMGD_LOSS_SOFTMAX) {
+        bmgdk::SoftmaxLaunchInfo info{};
+        EventPair ep{};
+        const bool timing = (h->cfg.flags & BMGD_FLAG_TIMING) != 0;
+        if (timing) {
+            int rc = take_events(h, &ep);
+            if (rc != BMGD_OK) return rc;
+            BMGD_CUDA(h, cudaEventRecord(ep.a, h->compute));
+        }
+        int rc = bmgdk::softmax_run(dx, dy, rows, h->cfg.p, h->cfg.C, h->base + h->lay.theta,
+                                   h->base + h->lay.softmax_scratch, reinterpret_cast<int*>(h->base + h->lay.status),
+                                   rounds, n, lr, seed, (h->cfg.flags & BMGD_FLAG_FIXED_PARTITION) ? 1 : 0,
+                                   h->timeout_ns, h->cfg.cluster_size, h->cfg.threads_per_cta, h->cfg.pipeline_depth,
+                                   h->sm_count, h->smem_optin, h->compute, &info);
+        if (rc != BMGD_OK) {
+            if (info.cuda_error) h->last_cuda = info.cuda_error;
+            if (timing) h->event_pool.push_back(ep);
+            return rc;
+        }
+        if (timing) {
+            BMGD_CUDA(h, cudaEventRecord(ep.b, h->compute));
+            h->kernel_events.push_back(ep);
+        }
+        const int64_t M = (rows + n - 1) / n;
+        h->stats.launches += info.launches;
+        h->stats.steps += (int64_t)rounds * M;
+        h->stats.sample_grads += (int64_t)rounds * rows;
+        h->stats.grid_ctas = info.grid_ctas;
+        h->stats.cluster_size = info.cluster_size;
+        h->stats.ctas_per_chain = info.grid_ctas;
+        h->stats.threads_per_cta = info.threads;
+        h->stats.pipeline_depth = info.depth;
+        h->stats.smem_bytes = info.smem;
+        h->stats.chains_in_flight = 1;
+        return BMGD_OK;
+    }
+    return run_glm(h, dx, dy, rows, rounds, n, lr, seed);
+}
+
+}  // namespace
+
+// ====================================================================== C ABI
+
+extern "C" {
+
+void bmgd_config_init(bmgd_config* cfg) {
+    if (!cfg) return;
+    std::memset(cfg, 0, sizeof *cfg);
+    cfg->loss = BMGD_LOSS_LINEAR;
+    cfg->dtype = BMGD_F32;
+    cfg->C = 1;
+    cfg->Rc = 1;
+    cfg->K = 1;
+    cfg->device = -1;
+}
+
+int bmgd_workspace_bytes(const bmgd_config* cfg, int64_t* bytes) {
+    if (!bytes) return BMGD_ERR_ARG;
+    int rc = validate(cfg);
+    if (rc != BMGD_OK) return rc;
+    *bytes = make_layout(cfg).total;
+    return BMGD_OK;
+}
+
+int bmgd_create(int64_t N, int32_t p, int32_t K, int32_t loss, bmgd_t** out) {
+    bmgd_config cfg;
+    bmgd_config_init(&cfg);
+    cfg.N = N; cfg.p = p; cfg.K = K; cfg.loss = loss;
+    return bmgd_create_ex(&cfg, out);
+}
+
+int bmgd_create_ex(const bmgd_config* cfg, bmgd_t** out) {
+    if (!out) return BMGD_ERR_ARG;
+    int rc = validate(cfg);
+    if (rc != BMGD_OK) return rc;
+    int dev = cfg->device;
+    if (dev < 0 && cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return BMGD_ERR_CUDA; }
+    DeviceGuard guard(dev);
+    if (!guard.ok) { cudaGetLastError(); return BMGD_ERR_CUDA; }
+
+    bmgd* h = new (std::nothrow) bmgd();
+    if (!h) return BMGD_ERR_ALLOC;
+    h->cfg = *cfg;
+    h->device = dev;
+    h->xb = elem_bytes_x(cfg->dtype);
+    h->tb = elem_bytes_theta(cfg->dtype);
+    h->yb = cfg->loss == BMGD_LOSS_SOFTMAX ? 4 : h->tb;
+    h->N0cap = (cfg->N + cfg->K - 1) / cfg->K;
+    h->num_slots = (cfg->flags & BMGD_FLAG_NO_SLOTS) ? 0 : 2;
+    h->timeout_ns = (uint64_t)((cfg->timeout_ms > 0 ? cfg->timeout_ms : 2000.0) * 1e6);
+    h->lay = make_layout(cfg);
+
+    auto fail = [&](int code) { bmgd_destroy(h); return code; };
+    cudaError_t e;
+    if ((e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess ||
+        (e = cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(BMGD_ERR_CUDA);
+    }
+    if (cfg->workspace) {
+        if (cfg->workspace_bytes < h->lay.total) return fail(BMGD_ERR_CAPACITY);
+        h->base = static_cast<unsigned char*>(cfg->workspace);
+    } else {
+        void* p = nullptr;
+        if (cudaMalloc(&p, (size_t)h->lay.total) != cudaSuccess) { cudaGetLastError(); return fail(BMGD_ERR_ALLOC); }
+        h->base = static_cast<unsigned char*>(p);
+        h->owns_base = true;
+    }
+    if (cfg->compute_stream) {
+        h->compute = static_cast<cudaStream_t>(cfg->compute_stream);
+    } else {
+        if (cudaStreamCreateWithFlags(&h->compute, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); return fail(BMGD_ERR_CUDA); }
+        h->owns_stream = true;
+    }
+    for (int s = 0; s < h->num_slots; ++s) {
+        if (cudaEventCreateWithFlags(&h->loaded[s], cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&h->freed[s], cudaEventDisableTiming) != cudaSuccess) {
+            cudaGetLastError();
+            return fail(BMGD_ERR_CUDA);
+        }
+    }
+    // theta = 0, packet area and status words = 0
+    if (cudaMemsetAsync(h->base + h->lay.theta, 0, (size_t)(h->lay.total - h->lay.theta), h->compute) != cudaSuccess ||
+        cudaStreamSynchronize(h->compute) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(BMGD_ERR_CUDA);
+    }
+    *out = h;
+    return BMGD_OK;
+}
+
+int bmgd_destroy(bmgd_t* h) {
+    if (!h) return BMGD_OK;
+    DeviceGuard guard(h->device);
+    if (h->compute) cudaStreamSynchronize(h->compute);
+    for (int s = 0; s < 2; ++s) {
+        if (h->loaded[s]) { cudaEventSynchronize(h->loaded[s]); cudaEventDestroy(h->loaded[s]); }
+        if (h->freed[s]) cudaEventDestroy(h->freed[s]);
+    }
+    auto kill = [](std::vector<EventPair>& v) {
+        for (EventPair& ep : v) { cudaEventDestroy(ep.a); cudaEventDestroy(ep.b); }
+        v.clear();
+    };
+    kill(h->kernel_events); kill(h->copy_events); kill(h->event_pool);
+    if (h->owns_stream && h->compute) cudaStreamDestroy(h->compute);
+    if (h->owns_base && h->base) cudaFree(h->base);
+    cudaGetLastError();
+    delete h;
+    return BMGD_OK;
+}
+
+int bmgd_load_buffer(bmgd_t* h, const void* host_x, const void* host_y, int64_t rows, void* stream, int32_t* slot) {
+    if (!h || !host_x || !host_y || !slot || rows <= 0) return BMGD_ERR_ARG;
+    if (h->num_slots == 0) return BMGD_ERR_STATE;
+    if (rows > h->N0cap) return BMGD_ERR_CAPACITY;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return cuda_fail(h, cudaErrorInvalidDevice);
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const int s = h->next_slot;
+    // the kernel that last read this slot must be done before the slot is overwritten
+    if (h->slot_has_data[s]) BMGD_CUDA(h, cudaStreamWaitEvent(cs, h->freed[s], 0));
+    EventPair ep{};
+    const bool timing = (h->cfg.flags & BMGD_FLAG_TIMING) != 0;
+    if (timing) {
+        int rc = take_events(h, &ep);
+        if (rc != BMGD_OK) return rc;
+        BMGD_CUDA(h, cudaEventRecord(ep.a, cs));
+    }
+    const size_t xbytes = (size_t)rows * h->cfg.p * h->xb, ybytes = (size_t)rows * h->yb;
+    BMGD_CUDA(h, cudaMemcpyAsync(h->base + h->lay.slot_x[s], host_x, xbytes, cudaMemcpyHostToDevice, cs));
+    BMGD_CUDA(h, cudaMemcpyAsync(h->base + h->lay.slot_y[s], host_y, ybytes, cudaMemcpyHostToDevice, cs));
+    if (timing) {
+        BMGD_CUDA(h, cudaEventRecord(ep.b, cs));
+        h->copy_events.push_back(ep);
+    }
+    BMGD_CUDA(h, cudaEventRecord(h->loaded[s], cs));
+    h->slot_rows[s] = rows;
+    h->slot_has_data[s] = true;
+    h->stats.h2d_bytes += (int64_t)(xbytes + ybytes);
+    h->next_slot = (s + 1) % h->num_slots;
+    *slot = s;
+    return BMGD_OK;
+}
+
+int bmgd_run_rounds(bmgd_t* h, int32_t slot, int32_t rounds, int32_t batch_size, double lr, uint64_t seed) {
+    if (!h) return BMGD_ERR_ARG;
+    if (slot < 0 || slot >= h->num_slots) return BMGD_ERR_ARG;
+    if (!h->slot_has_data[slot]) return BMGD_ERR_STATE;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return cuda_fail(h, cudaErrorInvalidDevice);
+    BMGD_CUDA(h, cudaStreamWaitEvent(h->compute, h->loaded[slot], 0));
+    int rc = run_any(h, h->base + h->lay.slot_x[slot], h->base + h->lay.slot_y[slot], h->slot_rows[slot], rounds,
+                     batch_size, lr, seed);
+    if (rc != BMGD_OK) return rc;
+    BMGD_CUDA(h, cudaEventRecord(h->freed[slot], h->compute));
+    return BMGD_OK;
+}
+
+int bmgd_run_rounds_resident(bmgd_t* h, const void* dev_x, const void* dev_y, int64_t rows, int32_t rounds,
+                             int32_t batch_size, double lr, uint64_t seed) {
+    if (!h || !dev_x || !dev_y) return BMGD_ERR_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return cuda_fail(h, cudaErrorInvalidDevice);
+    return run_any(h, dev_x, dev_y, rows, rounds, batch_size, lr, seed);
+}
+
+int bmgd_sync(bmgd_t* h) {
+    if (!h) return BMGD_ERR_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return cuda_fail(h, cudaErrorInvalidDevice);
+    BMGD_CUDA(h, cudaStreamSynchronize(h->compute));
+    for (int s = 0; s < h->num_slots; ++s)
+        if (h->slot_has_data[s]) BMGD_CUDA(h, cudaEventSynchronize(h->loaded[s]));
+    return check_status_word(h);
+}
+
+int bmgd_get_theta(bmgd_t* h, void* out_host, int64_t bytes) {
+    if (!h || !out_host) return BMGD_ERR_ARG;
+    const int64_t want = (int64_t)h->cfg.Rc * h->cfg.p * h->cfg.C * h->tb;
+    if (bytes != want) return BMGD_ERR_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return cuda_fail(h, cudaErrorInvalidDevice);
+    BMGD_CUDA(h, cudaStreamSynchronize(h->compute));
+    int rc = check_status_word(h);
+    BMGD_CUDA(h, cudaMemcpy(out_host, h->base + h->lay.theta, (size_t)want, cudaMemcpyDeviceToHost));
+    if (rc != BMGD_OK) return rc;
+    const int64_t cnt = want / h->tb;
+    bool finite = true;
+    if (h->tb == 8) { const double* v = static_cast<const double*>(out_host); for (int64_t i = 0; i < cnt; ++i) finite &= std::isfinite(v[i]); }
+    else { const float* v = static_cast<const float*>(out_host); for (int64_t i = 0; i < cnt; ++i) finite &= std::isfinite(v[i]); }
+    return finite ? BMGD_OK : BMGD_ERR_NONFINITE;
+}
+
+int bmgd_set_theta(bmgd_t* h, const void* host, int64_t bytes) {
+    if (!h || !host) return BMGD_ERR_ARG;
+    const int64_t want = (int64_t)h->cfg.Rc * h->cfg.p * h->cfg.C * h->tb;
+    if (bytes != want) return BMGD_ERR_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return cuda_fail(h, cudaErrorInvalidDevice);
+    BMGD_CUDA(h, cudaStreamSynchronize(h->compute));
+    BMGD_CUDA(h, cudaMemcpy(h->base + h->lay.theta, host, (size_t)want, cudaMemcpyHostToDevice));
+    return BMGD_OK;
+}
+
+int bmgd_get_stats(bmgd_t* h, bmgd_stats* out) {
+    if (!h || !out) return BMGD_ERR_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return cuda_fail(h, cudaErrorInvalidDevice);
+    BMGD_CUDA(h, cudaStreamSynchronize(h->compute));
+    int rc = drain_events(h, h->kernel_events, &h->stats.kernel_ms);
+    if (rc != BMGD_OK) return rc;
+    rc = drain_events(h, h->copy_events, &h->stats.h2d_ms);
+    if (rc != BMGD_OK) return rc;
+    *out = h->stats;
+    return check_status_word(h);
+}
+
+int bmgd_debug_perm(bmgd_t* h, uint64_t seed, uint32_t chain, uint32_t round, uint32_t N0, uint32_t* out_host) {
+    if (!h || !out_host || N0 == 0 || N0 > 0x7FFFFFFFu) return BMGD_ERR_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return cuda_fail(h, cudaErrorInvalidDevice);
+    uint32_t* d = nullptr;
+    if (cudaMalloc(&d, (size_t)N0 * 4) != cudaSuccess) { cudaGetLastError(); return BMGD_ERR_ALLOC; }
+    const int threads = 256;
+    const int blocks = (int)std::min<int64_t>(((int64_t)N0 + threads - 1) / threads, (int64_t)h->sm_count * 8);
+    bmgdk::perm_kernel<<<blocks, threads, 0, h->compute>>>(seed, chain, round, N0, d);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaMemcpyAsync(out_host, d, (size_t)N0 * 4, cudaMemcpyDeviceToHost, h->compute);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->compute);
+    cudaFree(d);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    return BMGD_OK;
+}
+
+const char* bmgd_strerror(int status) {
+    switch (status) {
+        case BMGD_OK: return "ok";
+        case BMGD_ERR_ARG: return "invalid argument";
+        case BMGD_ERR_ALLOC: return "out of memory";
+        case BMGD_ERR_CUDA: return "CUDA runtime error";
+        case BMGD_ERR_CAPACITY: return "more rows than the slot or workspace holds";
+        case BMGD_ERR_TIMEOUT: return "a device-side wait ran out of time";
+        case BMGD_ERR_NONFINITE: return "theta is not finite";
+        case BMGD_ERR_LAUNCH: return "the grid cannot be made co-resident";
+        case BMGD_ERR_UNIMPLEMENTED: return "no kernel for this loss, type or shape";
+        case BMGD_ERR_STATE: return "call out of order";
+        default: return "unknown status";
+    }
+}
+
+int bmgd_last_cuda_error(const bmgd_t* h) { return h ? h->last_cuda : 0; }
+
+int bmgd_version(void) { return kVersion; }
+
+}  // extern "C"

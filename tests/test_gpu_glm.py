@@ -1,0 +1,184 @@
+"""Parity of the fused least-squares / logistic step kernel with the CPU oracle, through the C ABI.
+
+Tolerances are the stated ones: relative L2 error of theta at most 1e-10 in fp64 and 1e-4 in fp32.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2312_08728_b200 import inputs
+from paper_2312_08728_b200.inputs import WORKLOADS, Workload, LOSS_LINEAR, LOSS_LOGISTIC, DTYPE_F32, DTYPE_F64
+
+from helpers import TOL, buffers_of, gpu_job, oracle_job, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+
+def check(w, buffers, chains=None, mode="slots", **shape):
+    theta, stats = gpu_job(w, buffers, mode=mode, **shape)
+    want = oracle_job(w, buffers, chains=chains)
+    worst = 0.0
+    for c, th in want.items():
+        err = rel_l2(theta[c], th)
+        worst = max(worst, err)
+        assert err <= TOL[w.dtype], (w.name, c, err, stats)
+    return theta, stats, worst
+
+
+def test_cfg1_full_job_fp64():
+    """Linear fp64, N=10,000, p=10, 5 buffers of 2,000, n=100, T=5, lr=0.05, 2 passes: every step of the job."""
+    w = WORKLOADS["cfg1"]
+    _, stats, _ = check(w, buffers_of(w))
+    assert stats["steps"] == 2 * 5 * 5 * 20
+    assert stats["sample_grads"] == 2 * 10_000 * 5
+
+
+@pytest.mark.parametrize("mode", ["slots", "resident"])
+def test_linear_fp32_chains(mode):
+    """cfg2's shape scaled down: several tiles per CTA and eight chains sharing the buffer."""
+    w = WORKLOADS["cfg2"].scaled(N=60_000, K=3, T=3, epochs=2, Rc=8)
+    check(w, buffers_of(w), mode=mode)
+
+
+def test_logistic_fp32_multi_cluster_ragged():
+    """cfg3's shape scaled down: p=200, n=4,096 with a ragged last mini-batch, all clusters on one chain."""
+    w = WORKLOADS["cfg3"].scaled(N=100_000, K=2, T=2, epochs=1)
+    assert w.N0 % w.n != 0
+    _, stats, _ = check(w, buffers_of(w))
+    assert stats["ctas_per_chain"] > stats["cluster_size"]  # the cross-cluster exchange ran
+
+
+def test_linear_fp32_p64_streaming_shape():
+    """cfg5's shape scaled down: p=64, n=2,048."""
+    w = WORKLOADS["cfg5"].scaled(N=300_000, K=3, T=2)
+    check(w, buffers_of(w))
+
+
+SMALL = Workload("small", LOSS_LOGISTIC, DTYPE_F32, N=6_000, p=40, K=2, n=500, T=2, lr=0.3, epochs=1, seed=3)
+
+
+@pytest.mark.parametrize("shape", [
+    dict(cluster_size=1, ctas_per_chain=1),
+    dict(cluster_size=1, ctas_per_chain=4),
+    dict(cluster_size=2, ctas_per_chain=2),
+    dict(cluster_size=2, ctas_per_chain=12),
+    dict(cluster_size=4, ctas_per_chain=4),
+    dict(cluster_size=4, ctas_per_chain=40),
+    dict(cluster_size=8, ctas_per_chain=8),
+    dict(cluster_size=8, ctas_per_chain=64),
+    dict(cluster_size=8, ctas_per_chain=8, threads_per_cta=512),
+    dict(cluster_size=8, ctas_per_chain=16, pipeline_depth=2),
+    dict(cluster_size=8, ctas_per_chain=16, pipeline_depth=16),
+])
+def test_launch_shapes_agree_with_the_oracle(shape):
+    _, stats, _ = check(SMALL, buffers_of(SMALL), mode="resident", **shape)
+    assert stats["cluster_size"] == shape["cluster_size"]
+    assert stats["ctas_per_chain"] == shape["ctas_per_chain"]
+
+
+def test_cluster_of_sixteen_if_the_device_allows_it():
+    from paper_2312_08728_b200.binding import BmgdError
+    try:
+        check(SMALL, buffers_of(SMALL), mode="resident", cluster_size=16, ctas_per_chain=16)
+    except BmgdError as e:  # non-portable cluster size: allowed to be refused, never to be wrong
+        assert e.status in (-7, -3), e
+
+
+@pytest.mark.parametrize("dtype,p", [(DTYPE_F32, 7), (DTYPE_F32, 33), (DTYPE_F64, 5), (DTYPE_F64, 31),
+                                     (DTYPE_F32, 4), (DTYPE_F32, 128), (DTYPE_F32, 132), (DTYPE_F32, 260),
+                                     (DTYPE_F32, 500), (DTYPE_F32, 1024), (DTYPE_F64, 130), (DTYPE_F64, 512)])
+def test_predictor_counts_including_unaligned_rows(dtype, p):
+    """Rows that are not 16-byte multiples take the element-wise copy path; every lane/chunk variant is reached."""
+    w = Workload("pvar", LOSS_LINEAR, dtype, N=1_500, p=p, K=1, n=128, T=2, lr=0.5 / p, epochs=1, rho=0.3, seed=p)
+    check(w, buffers_of(w), mode="resident")
+
+
+@pytest.mark.parametrize("N0,n", [(1, 1), (7, 1), (7, 7), (7, 100), (33, 32), (1000, 999), (1000, 1000), (257, 3)])
+def test_degenerate_sizes(N0, n):
+    """One row, one-row mini-batches, a full-batch round, a batch larger than the buffer, a one-row tail."""
+    w = Workload("edge", LOSS_LINEAR, DTYPE_F64, N=N0, p=6, K=1, n=n, T=3, lr=0.1, epochs=1, rho=0.5, seed=N0 + n)
+    check(w, buffers_of(w), mode="resident")
+    check(w, buffers_of(w), mode="resident", cluster_size=4, ctas_per_chain=8)
+
+
+def test_zero_rounds_is_a_no_op_and_runs_are_bitwise_reproducible():
+    from paper_2312_08728_b200.binding import Bmgd, FLAG_NO_SLOTS
+    w = SMALL
+    X, y = [t.cuda() for t in inputs.make_buffer(w, 0)]
+    outs = []
+    for rep in range(3):
+        with Bmgd(w.N, w.p, w.K, loss=w.loss, dtype=w.dtype, flags=FLAG_NO_SLOTS) as h:
+            h.run_rounds_resident(X, y, 0, w.n, w.lr, 1)
+            assert not h.get_theta().any()
+            h.run_rounds_resident(X, y, 3, w.n, w.lr, 1)
+            outs.append(h.get_theta())
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+
+
+def test_resume_from_saved_theta():
+    """theta handed from call to call equals theta saved, restored into a new handle and continued."""
+    from paper_2312_08728_b200.binding import Bmgd, FLAG_NO_SLOTS
+    w = SMALL
+    bufs = [tuple(t.cuda() for t in inputs.make_buffer(w, k)) for k in range(2)]
+    with Bmgd(w.N, w.p, w.K, loss=w.loss, dtype=w.dtype, flags=FLAG_NO_SLOTS) as h:
+        h.run_rounds_resident(*bufs[0], w.T, w.n, w.lr, 10)
+        mid = h.get_theta()
+        h.run_rounds_resident(*bufs[1], w.T, w.n, w.lr, 11)
+        end = h.get_theta()
+    with Bmgd(w.N, w.p, w.K, loss=w.loss, dtype=w.dtype, flags=FLAG_NO_SLOTS) as h2:
+        h2.set_theta(mid)
+        h2.run_rounds_resident(*bufs[1], w.T, w.n, w.lr, 11)
+        assert np.array_equal(h2.get_theta(), end)
+
+
+def test_fixed_partition_flag():
+    from paper_2312_08728_b200.binding import FLAG_FIXED_PARTITION
+    w = Workload("fixed", LOSS_LINEAR, DTYPE_F64, N=900, p=8, K=1, n=100, T=4, lr=0.1, epochs=1, rho=0.5, seed=5)
+    bufs = buffers_of(w)
+    theta, _ = gpu_job(w, bufs, mode="resident", flags=FLAG_FIXED_PARTITION)
+    want = oracle_job(w, bufs, fixed_partition=True)[0]
+    assert rel_l2(theta[0], want) <= 1e-10
+    assert rel_l2(theta[0], oracle_job(w, bufs)[0]) > 1e-8  # and it is not the fresh-partition result
+
+
+def test_errors_surface_as_codes():
+    from paper_2312_08728_b200.binding import Bmgd, BmgdError, ERR_CAPACITY, ERR_STATE, ERR_ARG, ERR_NONFINITE
+    w = SMALL.scaled(loss=LOSS_LINEAR)
+    X, y = inputs.make_buffer(w, 0)
+    with Bmgd(w.N, w.p, w.K, loss=w.loss, dtype=w.dtype) as h:
+        with pytest.raises(BmgdError) as e:
+            h.run_rounds(0, 1, 10, 0.1, 0)
+        assert e.value.status == ERR_STATE
+        big = torch.zeros(w.N0 + 1, w.p), torch.zeros(w.N0 + 1)
+        with pytest.raises(BmgdError) as e:
+            h.load_buffer(*big)
+        assert e.value.status == ERR_CAPACITY
+        with pytest.raises(BmgdError) as e:
+            h.run_rounds(5, 1, 10, 0.1, 0)
+        assert e.value.status == ERR_ARG
+        slot = h.load_buffer(X.pin_memory(), y.pin_memory())
+        h.run_rounds(slot, 2, w.n, 1e9, 0)  # absurd learning rate: theta blows up
+        with pytest.raises(BmgdError) as e:
+            h.get_theta()
+        assert e.value.status == ERR_NONFINITE
+
+
+@pytest.mark.parametrize("chains", [[0, 31, 63]])
+def test_cfg2_full_buffer_in_the_benchmarked_launch_shape(chains):
+    """One full cfg2 buffer (100,000 x 100, n=1,000, T=10) with all 64 chains in one launch, default shape:
+    three sampled chains against the oracle."""
+    w = WORKLOADS["cfg2"].scaled(N=100_000, K=1, epochs=1)
+    bufs = buffers_of(w)
+    theta, stats = gpu_job(w, bufs, mode="resident")
+    want = oracle_job(w, bufs, chains=chains)
+    for c in chains:
+        assert rel_l2(theta[c], want[c]) <= 1e-4, (c, stats)
+    assert stats["sample_grads"] == 64 * 10 * 100_000
+    # chains differ (distinct partitions) but all sit near the least-squares solution
+    assert np.abs(theta - 1.0).max() < 0.2 and np.unique(theta[:, 0]).size == 64
+
+
+def test_cfg3_one_full_buffer_default_shape():
+    """One full cfg3 buffer (1,000,000 x 200 logistic, n=4,096, 245 steps per round), two rounds."""
+    w = WORKLOADS["cfg3"].scaled(N=1_000_000, K=1, T=2, epochs=1)
+    check(w, buffers_of(w), mode="resident")
