@@ -150,6 +150,40 @@ int bmgd_run_rounds(bmgd_t* h, int32_t slot, int32_t rounds, int32_t batch_size,
 int bmgd_run_rounds_resident(bmgd_t* h, const void* dev_x, const void* dev_y, int64_t rows,
                              int32_t rounds, int32_t batch_size, double lr, uint64_t seed);
 
+/*
+ * The paper has no counterpart to this call; it exists for callers that must not allocate.
+ *
+ * Some programs cannot call cudaMalloc where they need this library: a plugin running inside
+ * another framework's memory budget, a service that fixed its device memory at start-up and
+ * runs with the allocator locked, a step of a latency-critical loop where the implicit
+ * device-wide synchronisation of an allocation is not acceptable.  bmgd_create_ex always
+ * needs device memory (its own or a caller's workspace) and host memory for the handle.
+ * This call needs neither: the scratch of the step kernel (the packets through which
+ * thread-block clusters exchange partial gradients, and the status words) sits in a fixed
+ * array of BMGD_NOALLOC_SCRATCH_BYTES that is part of the library image, so every GPU on
+ * which the library is used holds that much from the first use until the process exits.
+ * No cudaMalloc, cudaFree or other allocating routine is called.
+ *
+ * It runs `rounds` rounds over the buffer dev_x [rows][p], dev_y [rows] exactly as
+ * bmgd_run_rounds_resident does (same kernels, same shuffle, same launch-shape rules at their
+ * defaults) for the least-squares and logistic losses in BMGD_F32 or BMGD_F64, on the calling
+ * thread's current device, ordered on `stream` (a cudaStream_t; NULL = the legacy default
+ * stream).  dev_theta [Rc][p] is the caller's: it is read as the starting value and holds the
+ * result.  The call returns after the kernel has finished.
+ *
+ * Limits and sharing: p must not exceed BMGD_NOALLOC_MAX_P, else BMGD_ERR_CAPACITY is returned
+ * and nothing runs.  All calls on one GPU, from any thread or stream, use the same array; it
+ * keeps the contents of the previous call, so each call first clears the part it uses.  Two
+ * calls that overlap in time on one GPU would race on it: issue them one after the other.
+ * The first call on each device looks up the array's device address; make that first call
+ * outside any stream capture.
+ */
+#define BMGD_NOALLOC_MAX_P 256
+#define BMGD_NOALLOC_SCRATCH_BYTES (256 + 2 * 160 * BMGD_NOALLOC_MAX_P * 2 * 8)
+int bmgd_run_rounds_noalloc(const void* dev_x, const void* dev_y, int64_t rows, int32_t p, int32_t loss,
+                            int32_t dtype, int32_t Rc, void* dev_theta, int32_t rounds, int32_t batch_size,
+                            double lr, uint64_t seed, void* stream);
+
 /* Wait for everything issued on the compute stream; report a device-side error if one was raised. */
 int bmgd_sync(bmgd_t* h);
 

@@ -30,7 +30,7 @@ EXPORTS = (
     "bmgd_config_init", "bmgd_workspace_bytes", "bmgd_create", "bmgd_create_ex", "bmgd_destroy",
     "bmgd_load_buffer", "bmgd_run_rounds", "bmgd_run_rounds_resident", "bmgd_sync", "bmgd_get_theta",
     "bmgd_set_theta", "bmgd_get_stats", "bmgd_debug_perm", "bmgd_strerror", "bmgd_last_cuda_error",
-    "bmgd_version",
+    "bmgd_version", "bmgd_run_rounds_noalloc",
 )
 
 
@@ -102,6 +102,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.bmgd_strerror.argtypes = [ctypes.c_int]; L.bmgd_strerror.restype = ctypes.c_char_p
     L.bmgd_last_cuda_error.argtypes = [vp]
     L.bmgd_version.argtypes = []
+    L.bmgd_run_rounds_noalloc.argtypes = [vp, vp, i64, i32, i32, i32, i32, vp, i32, i32, dbl, u64, vp]
     for name in EXPORTS:
         if getattr(L, name).restype is None or name in ("bmgd_strerror",):
             continue
@@ -112,6 +113,33 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
 
 
 _NP_THETA = {DTYPE_F64: np.float64, DTYPE_F32: np.float32, DTYPE_BF16: np.float32}
+
+
+NOALLOC_MAX_P = 256
+
+
+def run_rounds_noalloc(dev_x: torch.Tensor, dev_y: torch.Tensor, theta: torch.Tensor, loss: int, dtype: int,
+                       rounds: int, batch_size: int, lr: float, seed: int,
+                       stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Allocation-free computation step: bmgd_run_rounds_noalloc on caller-held device tensors.
+
+    For callers that may not allocate device memory where they call this library (a fixed memory
+    budget, an allocator owned by someone else).  `theta` [Rc, p] lives on the device, is the
+    starting value and receives the result.  Nothing is allocated here either: the tensors are
+    passed as they are and must already be contiguous and on the current device.  Returns once the
+    kernel has finished; calls on one GPU must not overlap, they share one fixed scratch array.
+    """
+    for t in (dev_x, dev_y, theta):
+        if t.device.type != "cuda" or not t.is_contiguous():
+            raise ValueError("run_rounds_noalloc takes contiguous device tensors")
+    Rc, p = theta.shape
+    L = load_library()
+    s = stream.cuda_stream if stream is not None else None
+    rc = L.bmgd_run_rounds_noalloc(dev_x.data_ptr(), dev_y.data_ptr(), dev_x.shape[0], p, loss, dtype, Rc,
+                                   theta.data_ptr(), rounds, batch_size, float(lr),
+                                   int(seed) & 0xFFFFFFFFFFFFFFFF, s)
+    if rc != BMGD_OK:
+        raise BmgdError(rc, "bmgd_run_rounds_noalloc")
 
 
 class Bmgd:

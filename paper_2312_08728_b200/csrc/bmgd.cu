@@ -10,6 +10,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -668,6 +669,136 @@ int bmgd_debug_perm(bmgd_t* h, uint64_t seed, uint32_t chain, uint32_t round, ui
     if (e == cudaSuccess) e = cudaStreamSynchronize(h->compute);
     cudaFree(d);
     if (e != cudaSuccess) return cuda_fail(h, e);
+    return BMGD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free variant of the computation step.
+//
+// The step kernel needs scratch in global memory besides its inputs and outputs: the tagged
+// packets through which clusters exchange partial gradients, and two status words.  A handle
+// gets that scratch from cudaMalloc or from the caller's workspace.  Here it lives in a fixed
+// array that is part of the loaded library image instead.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[BMGD_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kNoallocMaxDevices = 64;
+void* g_noalloc_ptr[kNoallocMaxDevices];  // device address of g_noalloc_scratch, per device ordinal
+std::mutex g_noalloc_mutex;
+
+// In host code `g_noalloc_scratch` is only a handle for the symbol; the address a kernel can use
+// comes from cudaGetSymbolAddress, asked once per device with that device current.
+int noalloc_scratch_for_current_device(int dev, unsigned char** out) {
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+        if (e != cudaSuccess || !p) { cudaGetLastError(); return BMGD_ERR_CUDA; }
+        g_noalloc_ptr[dev] = p;
+    }
+    *out = static_cast<unsigned char*>(g_noalloc_ptr[dev]);
+    return BMGD_OK;
+}
+}  // namespace
+
+int bmgd_run_rounds_noalloc(const void* dev_x, const void* dev_y, int64_t rows, int32_t p, int32_t loss,
+                            int32_t dtype, int32_t Rc, void* dev_theta, int32_t rounds, int32_t batch_size,
+                            double lr, uint64_t seed, void* stream) {
+    if (!dev_x || !dev_y || !dev_theta) return BMGD_ERR_ARG;
+    if (loss != BMGD_LOSS_LINEAR && loss != BMGD_LOSS_LOGISTIC) return BMGD_ERR_UNIMPLEMENTED;
+    if (dtype != BMGD_F64 && dtype != BMGD_F32) return BMGD_ERR_UNIMPLEMENTED;
+    if (p <= 0 || Rc < 1 || Rc > 65536) return BMGD_ERR_ARG;
+    if (p > BMGD_NOALLOC_MAX_P) return BMGD_ERR_CAPACITY;  // the fixed scratch holds packets for at most this many predictors
+    if (rows <= 0 || rows > 0x7FFFFFFFll || rounds < 0 || batch_size <= 0 || !std::isfinite(lr)) return BMGD_ERR_ARG;
+    if (rounds == 0) return BMGD_OK;
+    int n = batch_size > rows ? (int)rows : batch_size;
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return BMGD_ERR_CUDA; }
+    if (dev < 0 || dev >= kNoallocMaxDevices) return BMGD_ERR_ARG;
+    unsigned char* scratch = nullptr;
+    int rc = noalloc_scratch_for_current_device(dev, &scratch);
+    if (rc != BMGD_OK) return rc;
+
+    // A handle on the stack, never registered anywhere: it only carries what the launch planner reads.
+    bmgd tmp;
+    bmgd_config_init(&tmp.cfg);
+    tmp.cfg.N = rows; tmp.cfg.p = p; tmp.cfg.K = 1; tmp.cfg.loss = loss; tmp.cfg.dtype = dtype; tmp.cfg.Rc = Rc;
+    tmp.device = dev;
+    tmp.tb = elem_bytes_theta(dtype);
+    if (cudaDeviceGetAttribute(&tmp.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&tmp.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return BMGD_ERR_CUDA;
+    }
+    const int tb = tmp.tb;
+    if (((uintptr_t)dev_x % tb) != 0 || ((uintptr_t)dev_y % tb) != 0 || ((uintptr_t)dev_theta % tb) != 0) return BMGD_ERR_ARG;
+    const bool aligned16 = ((int64_t)p * tb) % 16 == 0 && ((uintptr_t)dev_x % 16) == 0;
+    const GlmVariant* var = pick_variant(dtype, p, aligned16);
+    if (!var) return BMGD_ERR_UNIMPLEMENTED;
+    LaunchShape L{};
+    rc = plan_glm(&tmp, var, rows, n, &L);
+    if (rc != BMGD_OK) return rc;
+
+    const uint32_t M = (uint32_t)((rows + n - 1) / n);
+    const int chains_per_team = (Rc + L.nteams - 1) / L.nteams;
+    if ((uint64_t)chains_per_team * (uint64_t)rounds * M >= 0xFFFFFFF0ull) return BMGD_ERR_ARG;
+    if ((int64_t)L.nteams * L.cpc > kMaxClustersForExchange) return BMGD_ERR_LAUNCH;
+    const size_t packet_bytes = (size_t)2 * kMaxClustersForExchange * p * 2 * 8;
+    if (256 + packet_bytes > (size_t)BMGD_NOALLOC_SCRATCH_BYTES) return BMGD_ERR_CAPACITY;
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // The array still holds the packets and status of whoever called last: start from zero, so that
+    // tag 0 again means "nothing written yet".
+    if (cudaMemsetAsync(scratch, 0, 256 + packet_bytes, st) != cudaSuccess) { cudaGetLastError(); return BMGD_ERR_CUDA; }
+
+    GlmParams P{};
+    P.X = dev_x; P.y = dev_y;
+    P.theta = dev_theta;
+    P.status = reinterpret_cast<int*>(scratch);
+    P.ll = reinterpret_cast<unsigned long long*>(scratch + 256);
+    P.seed = seed;
+    P.timeout_ns = 2000000000ull;
+    P.alpha = lr;
+    P.N0 = (uint32_t)rows; P.n = (uint32_t)n; P.M = M; P.T = rounds; P.p = p;
+    P.loss = loss; P.Rc = Rc; P.S = L.S; P.cpc = L.cpc; P.nteams = L.nteams;
+    P.passes = L.passes; P.depth = L.depth; P.pitch = L.pitch;
+    P.ll_stride = p * 2;
+    P.tag_base = 0;
+    P.fixed_partition = 0;
+
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3((unsigned)(L.nteams * L.cpc * L.S), 1, 1);
+    lc.blockDim = dim3((unsigned)L.threads, 1, 1);
+    lc.dynamicSmemBytes = (size_t)L.smem;
+    lc.stream = st;
+    cudaLaunchAttribute at[2];
+    int na = 0;
+    if (L.S > 1) {
+        at[na].id = cudaLaunchAttributeClusterDimension;
+        at[na].val.clusterDim.x = (unsigned)L.S; at[na].val.clusterDim.y = 1; at[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    if (L.cpc > 1) {
+        at[na].id = cudaLaunchAttributeCooperative;
+        at[na].val.cooperative = 1;
+        ++na;
+    }
+    lc.attrs = at; lc.numAttrs = (unsigned)na;
+    cudaError_t e = cudaLaunchKernelEx(&lc, var->fn, P);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return (e == cudaErrorCooperativeLaunchTooLarge || e == cudaErrorLaunchOutOfResources) ? BMGD_ERR_LAUNCH : BMGD_ERR_CUDA;
+    }
+    // Wait for the kernel and read its status words back into a local: no other call could report them.
+    int status[2] = {0, 0};
+    if (cudaMemcpyAsync(status, scratch, sizeof status, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return BMGD_ERR_CUDA;
+    }
+    if (status[0] != 0) return status[0];
+    if (status[1] != 0) return BMGD_ERR_TIMEOUT;
     return BMGD_OK;
 }
 
