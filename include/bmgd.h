@@ -85,7 +85,8 @@ typedef struct bmgd_config {
     int32_t ctas_per_chain;
     int32_t threads_per_cta;  /* a multiple of 32, at most 1024 */
     int32_t pipeline_depth;   /* row-prefetch stages held in shared memory, 2..16 */
-    int32_t reserved[8];      /* must be zero */
+    int32_t subpasses_per_stage; /* a stage holds this many sweeps of the CTA over its rows: 1, 2, 4, ... 32 */
+    int32_t reserved[7];      /* must be zero */
 } bmgd_config;
 
 typedef struct bmgd_stats {
@@ -102,7 +103,7 @@ typedef struct bmgd_stats {
     int32_t pipeline_depth;
     int32_t smem_bytes;
     int32_t chains_in_flight;  /* chains worked on at the same time in the last launch */
-    int32_t reserved;
+    int32_t subpasses_per_stage;
 } bmgd_stats;
 
 /* Defaults: F32, linear, C = 1, Rc = 1, current device, two slots, library-owned memory. */

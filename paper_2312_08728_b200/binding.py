@@ -42,7 +42,7 @@ class BmgdConfig(ctypes.Structure):
         ("compute_stream", ctypes.c_void_p), ("timeout_ms", ctypes.c_double),
         ("cluster_size", ctypes.c_int32), ("ctas_per_chain", ctypes.c_int32),
         ("threads_per_cta", ctypes.c_int32), ("pipeline_depth", ctypes.c_int32),
-        ("reserved", ctypes.c_int32 * 8),
+        ("subpasses_per_stage", ctypes.c_int32), ("reserved", ctypes.c_int32 * 7),
     ]
 
 
@@ -52,7 +52,7 @@ class BmgdStats(ctypes.Structure):
         ("h2d_bytes", ctypes.c_int64), ("kernel_ms", ctypes.c_double), ("h2d_ms", ctypes.c_double),
         ("grid_ctas", ctypes.c_int32), ("cluster_size", ctypes.c_int32), ("ctas_per_chain", ctypes.c_int32),
         ("threads_per_cta", ctypes.c_int32), ("pipeline_depth", ctypes.c_int32), ("smem_bytes", ctypes.c_int32),
-        ("chains_in_flight", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("chains_in_flight", ctypes.c_int32), ("subpasses_per_stage", ctypes.c_int32),
     ]
 
     def as_dict(self):
@@ -151,7 +151,8 @@ class Bmgd:
 
     def __init__(self, N: int, p: int, K: int, loss: int = LOSS_LINEAR, dtype: int = DTYPE_F32, C: int = 1,
                  Rc: int = 1, device: int = 0, flags: int = 0, cluster_size: int = 0, ctas_per_chain: int = 0,
-                 threads_per_cta: int = 0, pipeline_depth: int = 0, timeout_ms: float = 0.0,
+                 threads_per_cta: int = 0, pipeline_depth: int = 0, subpasses_per_stage: int = 0,
+                 timeout_ms: float = 0.0,
                  use_torch_stream: bool = False):
         if not torch.cuda.is_available():
             raise RuntimeError("BMGD needs a CUDA device; there is no CPU path")
@@ -163,6 +164,7 @@ class Bmgd:
         cfg.device, cfg.flags = device, flags
         cfg.cluster_size, cfg.ctas_per_chain = cluster_size, ctas_per_chain
         cfg.threads_per_cta, cfg.pipeline_depth, cfg.timeout_ms = threads_per_cta, pipeline_depth, timeout_ms
+        cfg.subpasses_per_stage = subpasses_per_stage
         need = ctypes.c_int64()
         self._check(self._lib.bmgd_workspace_bytes(ctypes.byref(cfg), ctypes.byref(need)), "bmgd_workspace_bytes")
         self.device = torch.device("cuda", device)

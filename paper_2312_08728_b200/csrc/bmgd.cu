@@ -109,7 +109,7 @@ int validate(const bmgd_config* c) {
     }
     const int64_t N0 = (c->N + c->K - 1) / c->K;
     if (N0 > 0x7FFFFFFFll) return BMGD_ERR_ARG;
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < 7; ++i)
         if (c->reserved[i] != 0) return BMGD_ERR_ARG;
     if (c->cluster_size != 0 && c->cluster_size != 1 && c->cluster_size != 2 && c->cluster_size != 4 &&
         c->cluster_size != 8 && c->cluster_size != 16)
@@ -117,6 +117,10 @@ int validate(const bmgd_config* c) {
     if (c->threads_per_cta != 0 && (c->threads_per_cta % 32 != 0 || c->threads_per_cta < 256 || c->threads_per_cta > 1024))
         return BMGD_ERR_ARG;
     if (c->pipeline_depth != 0 && (c->pipeline_depth < 2 || c->pipeline_depth > 16)) return BMGD_ERR_ARG;
+    if (c->subpasses_per_stage != 0 && c->subpasses_per_stage != 1 && c->subpasses_per_stage != 2 &&
+        c->subpasses_per_stage != 4 && c->subpasses_per_stage != 8 && c->subpasses_per_stage != 16 &&
+        c->subpasses_per_stage != 32)
+        return BMGD_ERR_ARG;
     if (c->ctas_per_chain < 0) return BMGD_ERR_ARG;
     if (c->workspace && ((uintptr_t)c->workspace % kAlign) != 0) return BMGD_ERR_ARG;
     return BMGD_OK;
@@ -186,7 +190,7 @@ int floor_pow2(int v) {
 }
 
 struct LaunchShape {
-    int S, cpc, nteams, threads, depth, passes, pitch, smem;
+    int S, cpc, nteams, threads, depth, passes, rb, pitch, smem;
 };
 
 int max_active_clusters(bmgd* h, GlmKernel fn, int S, int threads, int smem, int* out) {
@@ -213,7 +217,7 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     L.threads = c.threads_per_cta ? std::min(c.threads_per_cta, var->max_threads())
                                   : ((c.Rc > 1 && var->max_threads() >= 512) ? 512 : 256);
     const int warps = L.threads / 32;
-    const int spp = warps * gpw;
+    const int spp = warps * gpw;  // rows a CTA works on at once (one sub-pass)
     L.pitch = (int)align_up((int64_t)c.p * eb, 16);
 
     // cluster size
@@ -226,22 +230,17 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     }
     L.S = S;
 
-    // fixed shared memory and a first guess at the depth, to ask the occupancy calculator
-    auto smem_for = [&](int depth) {
-        return bmgdk::glm_smem_plan(warps, gpw, depth, L.pitch, pcap, eb, S).total_bytes;
-    };
-    const int stage_bytes = spp * (L.pitch + 16);
-    int depth = c.pipeline_depth ? c.pipeline_depth : (int)std::min<int64_t>(16, std::max<int64_t>(3, (128 * 1024) / stage_bytes));
-    while (depth > 2 && smem_for(depth) > h->smem_optin) --depth;
-    if (smem_for(depth) > h->smem_optin) return BMGD_ERR_UNIMPLEMENTED;
-    L.depth = depth;
-    L.smem = smem_for(depth);
-
-    BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn, cudaFuncAttributeMaxDynamicSharedMemorySize, L.smem));
+    // How many clusters can be resident depends on shared memory, which depends on the ring; ask with
+    // the largest ring we would use (a smaller one can only admit more).
+    const int fixed_smem = bmgdk::glm_smem_plan(warps, gpw, 1, 0, L.pitch, pcap, eb, S).total_bytes;
+    const int ring_budget = std::min(h->smem_optin - fixed_smem, 160 * 1024);
+    if (ring_budget < spp * (L.pitch + 16)) return BMGD_ERR_UNIMPLEMENTED;
+    const int probe_smem = fixed_smem + ring_budget;
+    BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn, cudaFuncAttributeMaxDynamicSharedMemorySize, probe_smem));
     if (S > 8) BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
     int max_clusters = h->sm_count;
     if (S > 1) {
-        int rc = max_active_clusters(h, var->fn, S, L.threads, L.smem, &max_clusters);
+        int rc = max_active_clusters(h, var->fn, S, L.threads, probe_smem, &max_clusters);
         if (rc != BMGD_OK) return rc;
     }
     if (max_clusters < 1) return BMGD_ERR_LAUNCH;
@@ -265,12 +264,28 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     }
     const int G = L.cpc * S;
     const int rows_per_cta = (n + G - 1) / G;
-    L.passes = std::max(1, (rows_per_cta + spp - 1) / spp);
+    const int subpasses = std::max(1, (rows_per_cta + spp - 1) / spp);
+
+    // sub-passes per ring stage: fewer, larger stages amortise the per-stage bookkeeping
+    const int subpass_bytes = spp * (L.pitch + 16);
+    int rb = c.subpasses_per_stage ? c.subpasses_per_stage : var->lpr;
+    rb = std::min(rb, var->lpr);
+    rb = floor_pow2(std::max(1, std::min(rb, subpasses)));
+    const int stage_cap = c.subpasses_per_stage ? ring_budget / 2 : std::min(ring_budget / 3, 56 * 1024);
+    while (rb > 1 && rb * subpass_bytes > stage_cap) rb /= 2;
+    L.rb = rb;
+    L.passes = (subpasses + rb - 1) / rb;
+    const int stage_bytes = rb * subpass_bytes;
+    int depth = c.pipeline_depth ? c.pipeline_depth : std::max(2, (128 * 1024) / stage_bytes);
+    depth = std::min(depth, 16);
+    while (depth > 1 && depth * stage_bytes > ring_budget) --depth;
+    if (depth * stage_bytes > ring_budget) return BMGD_ERR_UNIMPLEMENTED;
+    L.depth = depth;
+    L.smem = bmgdk::glm_smem_plan(warps, gpw, rb, depth, L.pitch, pcap, eb, S).total_bytes;
     (void)rows;
     *out = L;
     return BMGD_OK;
 }
-
 
 int take_events(bmgd* h, EventPair* ep) {
     if (!h->event_pool.empty()) {
@@ -336,7 +351,8 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
     P.alpha = lr;
     P.N0 = (uint32_t)rows; P.n = (uint32_t)n; P.M = M; P.T = rounds; P.p = c.p;
     P.loss = c.loss; P.Rc = c.Rc; P.S = L.S; P.cpc = L.cpc; P.nteams = L.nteams;
-    P.passes = L.passes; P.depth = L.depth; P.pitch = L.pitch;
+    P.passes = L.passes; P.rb = L.rb; P.depth = L.depth; P.pitch = L.pitch;
+    P.q_full = (uint32_t)n / (uint32_t)(L.cpc * L.S); P.r_full = (uint32_t)n % (uint32_t)(L.cpc * L.S);
     P.ll_stride = c.p * 2;
     P.tag_base = (uint32_t)h->tag_base;
     P.fixed_partition = (c.flags & BMGD_FLAG_FIXED_PARTITION) ? 1 : 0;
@@ -389,6 +405,7 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
     h->stats.ctas_per_chain = L.cpc * L.S;
     h->stats.threads_per_cta = L.threads;
     h->stats.pipeline_depth = L.depth;
+    h->stats.subpasses_per_stage = L.rb;
     h->stats.smem_bytes = L.smem;
     h->stats.chains_in_flight = L.nteams;
     return BMGD_OK;
@@ -762,7 +779,8 @@ int bmgd_run_rounds_noalloc(const void* dev_x, const void* dev_y, int64_t rows, 
     P.alpha = lr;
     P.N0 = (uint32_t)rows; P.n = (uint32_t)n; P.M = M; P.T = rounds; P.p = p;
     P.loss = loss; P.Rc = Rc; P.S = L.S; P.cpc = L.cpc; P.nteams = L.nteams;
-    P.passes = L.passes; P.depth = L.depth; P.pitch = L.pitch;
+    P.passes = L.passes; P.rb = L.rb; P.depth = L.depth; P.pitch = L.pitch;
+    P.q_full = (uint32_t)n / (uint32_t)(L.cpc * L.S); P.r_full = (uint32_t)n % (uint32_t)(L.cpc * L.S);
     P.ll_stride = p * 2;
     P.tag_base = 0;
     P.fixed_partition = 0;
@@ -819,6 +837,15 @@ const char* bmgd_strerror(int status) {
 }
 
 int bmgd_last_cuda_error(const bmgd_t* h) { return h ? h->last_cuda : 0; }
+
+#ifdef BMGD_TRACE
+// Debug build only: copy out the clock stamps CTA 0 took at the phase boundaries of its first steps.
+int bmgd_debug_trace(long long* out_host, int count) {
+    if (!out_host || count <= 0 || count > bmgdk::kTraceSteps * bmgdk::kTracePhases) return BMGD_ERR_ARG;
+    cudaError_t e = cudaMemcpyFromSymbol(out_host, bmgdk::g_trace, sizeof(long long) * (size_t)count);
+    return e == cudaSuccess ? BMGD_OK : BMGD_ERR_CUDA;
+}
+#endif
 
 int bmgd_version(void) { return kVersion; }
 

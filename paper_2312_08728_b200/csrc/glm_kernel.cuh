@@ -7,7 +7,9 @@
 //
 // Per step, in every CTA:
 //   1. rows pi(j) of this CTA's share were prefetched into a shared-memory ring by cp.async,
-//      several passes ahead (rows do not depend on theta, the shuffle is stateless);
+//      several stages ahead (rows do not depend on theta, the shuffle is stateless); each lane
+//      evaluates pi for one row and the warp shares the 32 results by shuffle; the copies for a
+//      later stage are issued while the CTA would otherwise wait at a barrier;
 //   2. a group of LPR lanes owns one row: x.theta by an LPR-lane butterfly, the residual
 //      (x.theta - y, or sigmoid(x.theta) - y), then g += r * x with x still in registers, so a
 //      row is read from HBM once and from shared memory once;
@@ -51,8 +53,10 @@ struct GlmParams {
     int S;                // cluster size
     int cpc;              // clusters per chain
     int nteams;
-    int passes;           // passes per step: ceil(ceil(n/G) / rows per pass)
-    int depth;            // ring stages
+    int passes;           // ring stages per step
+    int rb;               // sub-passes per ring stage (a power of two, at most LPR)
+    int depth;            // ring stages in flight
+    uint32_t q_full, r_full;  // n / G and n % G: how a full mini-batch is dealt to the G CTAs
     int pitch;            // bytes between rows in the ring (multiple of 16)
     int ll_stride;        // packets per cluster slot
     uint32_t tag_base;
@@ -87,7 +91,8 @@ __device__ __forceinline__ void cp_async_wait_pending(int n) {
         case 11: asm volatile("cp.async.wait_group 11;" ::: "memory"); break;
         case 12: asm volatile("cp.async.wait_group 12;" ::: "memory"); break;
         case 13: asm volatile("cp.async.wait_group 13;" ::: "memory"); break;
-        default: asm volatile("cp.async.wait_group 14;" ::: "memory"); break;
+        case 14: asm volatile("cp.async.wait_group 14;" ::: "memory"); break;
+        default: asm volatile("cp.async.wait_group 15;" ::: "memory"); break;
     }
 }
 
@@ -158,10 +163,10 @@ struct GlmSmemPlan {
     int total_bytes;
 };
 
-__host__ __device__ inline GlmSmemPlan glm_smem_plan(int warps, int gpw, int depth, int pitch, int pcap,
+__host__ __device__ inline GlmSmemPlan glm_smem_plan(int warps, int gpw, int rb, int depth, int pitch, int pcap,
                                                      int elem_bytes, int S) {
     GlmSmemPlan s;
-    s.warp_stage_bytes = gpw * pitch + gpw * 16;
+    s.warp_stage_bytes = rb * gpw * (pitch + 16);
     s.ring_bytes = warps * depth * s.warp_stage_bytes;
     s.gpart_off = s.ring_bytes;
     s.cpart_off = s.gpart_off + warps * gpw * pcap * elem_bytes;
@@ -169,6 +174,19 @@ __host__ __device__ inline GlmSmemPlan glm_smem_plan(int warps, int gpw, int dep
     s.total_bytes = s.gfin_off + pcap * elem_bytes;
     return s;
 }
+
+#ifdef BMGD_TRACE
+// Debug build only: clock stamps of CTA 0 at the phase boundaries of its first steps.
+constexpr int kTraceSteps = 64, kTracePhases = 8;
+__device__ long long g_trace[kTraceSteps * kTracePhases];
+#define BMGD_STAMP(ph)                                                                              \
+    do {                                                                                            \
+        if (blockIdx.x == 0 && threadIdx.x == 0 && step_count < (uint32_t)kTraceSteps)              \
+            g_trace[step_count * kTracePhases + (ph)] = clock64();                                  \
+    } while (0)
+#else
+#define BMGD_STAMP(ph) do { } while (0)
+#endif
 
 // ---------------------------------------------------------------- the kernel
 
@@ -178,9 +196,28 @@ __host__ __device__ constexpr int glm_max_threads() {
     return (sizeof(T) == 8 || KCH * VEC >= 32) ? 256 : 512;
 }
 
+// How mini-batch rows [lo, lo+nm) are dealt to CTA g of G: a contiguous run of `cnt` rows from lo+a.
+struct RowShare {
+    uint32_t lo, a, cnt;
+};
+__device__ __forceinline__ RowShare row_share(uint32_t m, uint32_t n, uint32_t N0, uint32_t g, uint32_t G,
+                                              uint32_t q_full, uint32_t r_full) {
+    RowShare s;
+    s.lo = m * n;
+    const uint32_t nm = min(n, N0 - s.lo);
+    uint32_t q = q_full, r = r_full;
+    if (nm != n) { q = nm / G; r = nm % G; }
+    s.a = g * q + min(g, r);
+    s.cnt = q + (g < r ? 1u : 0u);
+    return s;
+}
+
 // T: float or double.  VEC: elements per copy chunk (16 bytes worth, or 1 when rows are not
 // 16-byte multiples).  LPR: lanes per row.  KCH: chunks per lane.  A row has at most
 // LPR*KCH*VEC predictors.
+//
+// Row slots of a CTA within one step are numbered u = (sp*W + warp)*GPW + grp, sp = sub-pass:
+// in sub-pass sp every warp works on GPW rows at once.  A ring stage holds `rb` sub-passes.
 template <typename T, int VEC, int LPR, int KCH>
 __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(const GlmParams P) {
     constexpr int GPW = 32 / LPR;            // row groups per warp
@@ -189,6 +226,7 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
     constexpr int FPT = (PCAP + 255) / 256;  // features per thread in the reductions (blockDim >= 256)
     constexpr int CB = VEC * (int)sizeof(T); // copy chunk bytes
     constexpr int NW = Words<T>::N;
+    constexpr uint32_t kNoRow = 0xFFFFFFFFu;
 
     extern __shared__ __align__(16) unsigned char smem[];
 
@@ -200,13 +238,13 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
     const int cluster_id = blockIdx.x / S;
     const int team = cluster_id / cpc, kc = cluster_id % cpc;
     const int g = kc * S + rank;
-    const int spp = W * GPW;  // rows per pass
     const int p = P.p, nchunks = p / VEC;
     const uint32_t N0 = P.N0, n = P.n, M = P.M;
-    const int T_rounds = P.T, passes = P.passes, D = P.depth, pitch = P.pitch;
+    const int T_rounds = P.T, passes = P.passes, RB = P.rb, D = P.depth, pitch = P.pitch;
 
-    const GlmSmemPlan plan = glm_smem_plan(W, GPW, D, pitch, PCAP, (int)sizeof(T), S);
+    const GlmSmemPlan plan = glm_smem_plan(W, GPW, RB, D, pitch, PCAP, (int)sizeof(T), S);
     unsigned char* my_ring = smem + (size_t)warp * D * plan.warp_stage_bytes;
+    const int y_off = RB * GPW * pitch;  // y values follow the rows of a warp's stage
     T* gpart = reinterpret_cast<T*>(smem + plan.gpart_off);
     T* cpart = reinterpret_cast<T*>(smem + plan.cpart_off);
     T* gfin = reinterpret_cast<T*>(smem + plan.gfin_off);
@@ -224,34 +262,39 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
         cluster_wait_acquire();
     }
 
-    // ---- prefetch cursor: runs D-1 passes ahead of the compute cursor
-    int pf_ci = 0, pf_t = 0, pf_pass = 0, pf_stage = 0;
+    // ---- prefetch cursor: runs D stages ahead of the compute cursor
+    int pf_ci = 0, pf_t = 0, pf_sidx = 0, pf_slot = 0;
     uint32_t pf_m = 0;
+    uint32_t pf_rows = kNoRow;  // this lane's row of the current batch of 32 row slots
     long long issued = 0;
     RoundKeys pfk = round_keys(P.seed, (uint32_t)team, 0u);
+    RowShare pfs = row_share(0u, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full);
 
     auto issue_one = [&]() {
         if (issued < nstages) {
-            const uint32_t lo = pf_m * n;
-            const uint32_t nm = min(n, N0 - lo);
-            const uint32_t a = (uint32_t)(((unsigned long long)g * nm) / (unsigned)G);
-            const uint32_t b = (uint32_t)(((unsigned long long)(g + 1) * nm) / (unsigned)G);
-            const uint32_t u = (uint32_t)(pf_pass * spp + warp * GPW + grp);
-            if (u < b - a) {
-                const uint32_t row = perm_index(lo + a + u, dom, pfk);
-                const unsigned char* src = Xb + (size_t)row * row_bytes;
-                unsigned char* stage = my_ring + (size_t)pf_stage * plan.warp_stage_bytes;
-                const uint32_t dst = smem_u32(stage + grp * pitch);
-#pragma unroll
-                for (int k = 0; k < KCH; ++k) {
-                    const int c = sub + k * LPR;
-                    if (c < nchunks) cp_async<CB>(dst + c * CB, src + (size_t)c * CB);
+            unsigned char* stage = my_ring + (size_t)pf_slot * plan.warp_stage_bytes;
+            for (int r = 0; r < RB; ++r) {
+                const int sp = pf_sidx * RB + r;
+                const int bi = sp & (LPR - 1);
+                if (bi == 0) {  // a new batch: lane l takes sub-pass sp + l/GPW, group l%GPW
+                    const uint32_t u = ((uint32_t)(sp + lane / GPW) * (uint32_t)W + (uint32_t)warp) * GPW + (lane % GPW);
+                    pf_rows = (u < pfs.cnt) ? perm_index(pfs.lo + pfs.a + u, dom, pfk) : kNoRow;
                 }
-                if (sub == 0) cp_async<(int)sizeof(T)>(smem_u32(stage + GPW * pitch + grp * 16), yb + row);
+                const uint32_t row = __shfl_sync(0xFFFFFFFFu, pf_rows, bi * GPW + grp);
+                if (row != kNoRow) {
+                    const unsigned char* src = Xb + (size_t)row * row_bytes;
+                    const int slot_row = r * GPW + grp;
+                    const uint32_t dst = smem_u32(stage + slot_row * pitch);
+#pragma unroll
+                    for (int k = 0; k < KCH; ++k) {
+                        const int c = sub + k * LPR;
+                        if (c < nchunks) cp_async<CB>(dst + c * CB, src + (size_t)c * CB);
+                    }
+                    if (sub == 0) cp_async<(int)sizeof(T)>(smem_u32(stage + y_off + slot_row * 16), yb + row);
+                }
             }
-            // advance
-            if (++pf_pass == passes) {
-                pf_pass = 0;
+            if (++pf_sidx == passes) {
+                pf_sidx = 0;
                 if (++pf_m == M) {
                     pf_m = 0;
                     if (++pf_t == T_rounds) { pf_t = 0; ++pf_ci; }
@@ -259,16 +302,18 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                         pfk = round_keys(P.seed, (uint32_t)(team + pf_ci * P.nteams),
                                          P.fixed_partition ? 0u : (uint32_t)pf_t);
                 }
+                pfs = row_share(pf_m, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full);
             }
-            if (++pf_stage == D) pf_stage = 0;
+            if (++pf_slot == D) pf_slot = 0;
         }
         cp_async_commit();
         ++issued;
+        __syncwarp();  // lanes walked the cycle for different lengths: meet again before any aligned barrier
     };
 
-    for (int s = 0; s < D - 1; ++s) issue_one();
+    for (int s = 0; s < D; ++s) issue_one();
 
-    int cs_stage = 0;        // ring stage the compute cursor reads next
+    int cs_slot = 0;         // ring slot the compute cursor reads next
     uint32_t step_count = 0; // steps this team has finished in this launch
     bool aborted = false;
     const bool logistic = (P.loss == 1);
@@ -287,67 +332,72 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
 
         for (int t = 0; t < T_rounds; ++t) {
             for (uint32_t m = 0; m < M; ++m) {
-                const uint32_t lo = m * n;
-                const uint32_t nm = min(n, N0 - lo);
-                const uint32_t a = (uint32_t)(((unsigned long long)g * nm) / (unsigned)G);
-                const uint32_t b = (uint32_t)(((unsigned long long)(g + 1) * nm) / (unsigned)G);
-                const uint32_t cnt = b - a;
+                const RowShare sh = row_share(m, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full);
+                const uint32_t nm = min(n, N0 - sh.lo);
+                BMGD_STAMP(0);
 
                 T gacc[NV];
 #pragma unroll
                 for (int i = 0; i < NV; ++i) gacc[i] = T(0);
 
-                for (int pass = 0; pass < passes; ++pass) {
-                    cp_async_wait_pending(D - 2);
+                for (int sidx = 0; sidx < passes; ++sidx) {
+                    cp_async_wait_pending(D - 1);
                     __syncwarp();
-                    issue_one();
+                    const unsigned char* stage = my_ring + (size_t)cs_slot * plan.warp_stage_bytes;
+                    if (++cs_slot == D) cs_slot = 0;
 
-                    const unsigned char* stage = my_ring + (size_t)cs_stage * plan.warp_stage_bytes;
-                    if (++cs_stage == D) cs_stage = 0;
-                    const uint32_t u = (uint32_t)(pass * spp + warp * GPW + grp);
-                    const bool valid = u < cnt;
+                    for (int r = 0; r < RB; ++r) {
+                        const uint32_t u = ((uint32_t)(sidx * RB + r) * (uint32_t)W + (uint32_t)warp) * GPW + grp;
+                        const bool valid = u < sh.cnt;
+                        const int slot_row = r * GPW + grp;
 
-                    T x[NV];
-                    const unsigned char* rowp = stage + grp * pitch;
+                        T x[NV];
+                        const unsigned char* rowp = stage + slot_row * pitch;
 #pragma unroll
-                    for (int k = 0; k < KCH; ++k) {
-                        const int c = sub + k * LPR;
-                        if (valid && c < nchunks) {
-                            if constexpr (CB == 16 && sizeof(T) == 4) {
-                                const float4 v = *reinterpret_cast<const float4*>(rowp + c * 16);
-                                x[k * VEC + 0] = v.x; x[k * VEC + 1] = v.y; x[k * VEC + 2] = v.z; x[k * VEC + 3] = v.w;
-                            } else if constexpr (CB == 16) {
-                                const double2 d = *reinterpret_cast<const double2*>(rowp + c * 16);
-                                x[k * VEC + 0] = d.x; x[k * VEC + 1] = d.y;
+                        for (int k = 0; k < KCH; ++k) {
+                            const int c = sub + k * LPR;
+                            if (valid && c < nchunks) {
+                                if constexpr (CB == 16 && sizeof(T) == 4) {
+                                    const float4 v = *reinterpret_cast<const float4*>(rowp + c * 16);
+                                    x[k * VEC + 0] = v.x; x[k * VEC + 1] = v.y; x[k * VEC + 2] = v.z; x[k * VEC + 3] = v.w;
+                                } else if constexpr (CB == 16) {
+                                    const double2 d = *reinterpret_cast<const double2*>(rowp + c * 16);
+                                    x[k * VEC + 0] = d.x; x[k * VEC + 1] = d.y;
+                                } else {
+                                    x[k] = *reinterpret_cast<const T*>(rowp + c * CB);
+                                }
                             } else {
-                                x[k] = *reinterpret_cast<const T*>(rowp + c * CB);
+#pragma unroll
+                                for (int e = 0; e < VEC; ++e) x[k * VEC + e] = T(0);
                             }
-                        } else {
-#pragma unroll
-                            for (int e = 0; e < VEC; ++e) x[k * VEC + e] = T(0);
                         }
-                    }
-                    T part[VEC];
+                        T part[VEC];
 #pragma unroll
-                    for (int e = 0; e < VEC; ++e) part[e] = T(0);
+                        for (int e = 0; e < VEC; ++e) part[e] = T(0);
 #pragma unroll
-                    for (int k = 0; k < KCH; ++k)
+                        for (int k = 0; k < KCH; ++k)
 #pragma unroll
-                        for (int e = 0; e < VEC; ++e) part[e] = fma(x[k * VEC + e], th[k * VEC + e], part[e]);
-                    T dot = part[0];
+                            for (int e = 0; e < VEC; ++e) part[e] = fma(x[k * VEC + e], th[k * VEC + e], part[e]);
+                        T dot = part[0];
 #pragma unroll
-                    for (int e = 1; e < VEC; ++e) dot += part[e];
+                        for (int e = 1; e < VEC; ++e) dot += part[e];
 #pragma unroll
-                    for (int off = LPR / 2; off > 0; off >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, off);
+                        for (int off = LPR / 2; off > 0; off >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, off);
 
-                    T r = T(0);
-                    if (valid) {
-                        const T yv = *reinterpret_cast<const T*>(stage + GPW * pitch + grp * 16);
-                        r = (logistic ? sigmoid_of(dot) : dot) - yv;
-                    }
+                        T res = T(0);
+                        if (valid) {
+                            const T yv = *reinterpret_cast<const T*>(stage + y_off + slot_row * 16);
+                            res = (logistic ? sigmoid_of(dot) : dot) - yv;
+                        }
 #pragma unroll
-                    for (int i = 0; i < NV; ++i) gacc[i] = fma(r, x[i], gacc[i]);
+                        for (int i = 0; i < NV; ++i) gacc[i] = fma(res, x[i], gacc[i]);
+                    }
+                    if (sidx + 1 < passes) {  // refill the slot just read; the last one of a step waits for a barrier
+                        __syncwarp();
+                        issue_one();
+                    }
                 }
+                BMGD_STAMP(1);
 
                 // ---- sum the group partials of this CTA in fixed order
                 {
@@ -359,7 +409,13 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                         for (int e = 0; e < VEC; ++e) gp[c * VEC + e] = gacc[k * VEC + e];
                     }
                 }
+                if (S == 1 && cpc == 1) {
+                    __syncwarp();
+                    issue_one();
+                }
                 __syncthreads();
+                BMGD_STAMP(2);
+                const int spp = W * GPW;
                 T tot[FPT];
 #pragma unroll
                 for (int i = 0; i < FPT; ++i) {
@@ -378,6 +434,7 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                     }
                     tot[i] = (s0 + s1) + (s2 + s3);
                 }
+                BMGD_STAMP(3);
 
                 const int parity = (int)(step_count & 1u);
 
@@ -392,7 +449,9 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                             for (int peer = 0; peer < S; ++peer)
                                 st_cluster(map_to_cta(mine + f * (uint32_t)sizeof(T), (uint32_t)peer), tot[i]);
                     }
+                    __syncwarp();
                     cluster_arrive_release();
+                    issue_one();  // the copies for a later stage go out while the barrier completes
                     cluster_wait_acquire();
 #pragma unroll
                     for (int i = 0; i < FPT; ++i) {
@@ -403,6 +462,7 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                         tot[i] = s;
                     }
                 }
+                BMGD_STAMP(4);
 
                 // ---- across clusters: tagged packets through global memory
                 if (cpc > 1) {
@@ -419,6 +479,7 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                                           ((unsigned long long)tag << 32) | Words<T>::get(tot[i], w));
                         }
                     }
+                    if (S == 1) issue_one();
 #pragma unroll
                     for (int i = 0; i < FPT; ++i) {
                         const int f = tid + i * nthreads;
@@ -465,6 +526,7 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                         tot[i] = s;
                     }
                 }
+                BMGD_STAMP(5);
 
                 // ---- everyone updates its own copy of theta
 #pragma unroll
@@ -474,6 +536,7 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                 }
                 // a thread that gave up tells the rest of its CTA, so that no one else waits out its own budget
                 aborted = __syncthreads_or(aborted ? 1 : 0) != 0;
+                BMGD_STAMP(6);
                 const T scale = (T)(P.alpha / (double)nm);
 #pragma unroll
                 for (int k = 0; k < KCH; ++k) {
@@ -481,6 +544,7 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
 #pragma unroll
                     for (int e = 0; e < VEC; ++e) th[k * VEC + e] -= scale * gfin[c * VEC + e];
                 }
+                BMGD_STAMP(7);
                 ++step_count;
             }
         }
