@@ -51,6 +51,7 @@ def parse_args():
     ap.add_argument("--ctas-per-chain", type=int, default=0)
     ap.add_argument("--threads", type=int, default=0)
     ap.add_argument("--depth", type=int, default=0)
+    ap.add_argument("--subpasses", type=int, default=0, help="sub-passes per ring stage")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
@@ -250,7 +251,7 @@ def run_ours(args, w):
     host = [inputs.make_buffer(w, k) for k in range(nb)]
     seed0 = w.seed + rank * 1_000_003
     shape = dict(cluster_size=args.cluster_size, ctas_per_chain=args.ctas_per_chain, threads_per_cta=args.threads,
-                 pipeline_depth=args.depth)
+                 pipeline_depth=args.depth, subpasses_per_stage=args.subpasses)
     sg_per_step = [x.shape[0] * w.T * w.Rc for x, _ in host]
 
     # ---- device-resident measurement
@@ -343,7 +344,8 @@ def run_ours(args, w):
                 "kernel_ms_per_launch": kdur * 1e3, "algorithmic_bytes_per_launch": bytes_per_launch,
                 "us_per_minibatch_step": 1e3 * kernel_ms / max(1, (s1["steps"] - s0["steps"]) / w.Rc),
                 "launch_shape": {k: s1[k] for k in ("grid_ctas", "cluster_size", "ctas_per_chain", "threads_per_cta",
-                                                    "pipeline_depth", "smem_bytes", "chains_in_flight")}}
+                                                    "pipeline_depth", "subpasses_per_stage", "smem_bytes",
+                                                    "chains_in_flight")}}
     if w.name == "cfg2":
         roofline["note"] = ("one 40 MB buffer is re-read Rc*T = 640 times per launch and stays in the 126 MB L2, "
                             "so algorithmic bytes per second may exceed the HBM peak; DRAM traffic is in `traffic`")

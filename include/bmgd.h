@@ -83,8 +83,8 @@ typedef struct bmgd_config {
      * (a multiple of cluster_size); the rows of a mini-batch are split among them. */
     int32_t cluster_size;     /* CTAs per thread-block cluster: 1, 2, 4, 8 or 16 */
     int32_t ctas_per_chain;
-    int32_t threads_per_cta;  /* a multiple of 32, at most 1024 */
-    int32_t pipeline_depth;   /* row-prefetch stages held in shared memory, 2..16 */
+    int32_t threads_per_cta;  /* 256, 512 or 1024 */
+    int32_t pipeline_depth;   /* row-prefetch stages held in shared memory: 2, 3 or 4 */
     int32_t subpasses_per_stage; /* a stage holds this many sweeps of the CTA over its rows: 1, 2, 4, ... 32 */
     int32_t reserved[7];      /* must be zero */
 } bmgd_config;

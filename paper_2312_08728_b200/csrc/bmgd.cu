@@ -114,9 +114,9 @@ int validate(const bmgd_config* c) {
     if (c->cluster_size != 0 && c->cluster_size != 1 && c->cluster_size != 2 && c->cluster_size != 4 &&
         c->cluster_size != 8 && c->cluster_size != 16)
         return BMGD_ERR_ARG;
-    if (c->threads_per_cta != 0 && (c->threads_per_cta % 32 != 0 || c->threads_per_cta < 256 || c->threads_per_cta > 1024))
+    if (c->threads_per_cta != 0 && c->threads_per_cta != 256 && c->threads_per_cta != 512 && c->threads_per_cta != 1024)
         return BMGD_ERR_ARG;
-    if (c->pipeline_depth != 0 && (c->pipeline_depth < 2 || c->pipeline_depth > 16)) return BMGD_ERR_ARG;
+    if (c->pipeline_depth != 0 && (c->pipeline_depth < 2 || c->pipeline_depth > 4)) return BMGD_ERR_ARG;
     if (c->subpasses_per_stage != 0 && c->subpasses_per_stage != 1 && c->subpasses_per_stage != 2 &&
         c->subpasses_per_stage != 4 && c->subpasses_per_stage != 8 && c->subpasses_per_stage != 16 &&
         c->subpasses_per_stage != 32)
@@ -158,26 +158,25 @@ struct GlmVariant {
     int max_threads() const { return maxt; }
 };
 
-template <typename T>
+template <typename T, bool LG>
 const GlmVariant* glm_variants(bool aligned16, int* count) {
     constexpr int V = 16 / (int)sizeof(T);
-    static const GlmVariant wide[] = {
-        {bmgdk::glm_kernel<T, V, 8, 1>, V, 8, 1, bmgdk::glm_max_threads<T, V, 1>()},  {bmgdk::glm_kernel<T, V, 8, 2>, V, 8, 2, bmgdk::glm_max_threads<T, V, 2>()},
-        {bmgdk::glm_kernel<T, V, 8, 4>, V, 8, 4, bmgdk::glm_max_threads<T, V, 4>()},  {bmgdk::glm_kernel<T, V, 8, 8>, V, 8, 8, bmgdk::glm_max_threads<T, V, 8>()},
-        {bmgdk::glm_kernel<T, V, 16, 8>, V, 16, 8, bmgdk::glm_max_threads<T, V, 8>()}, {bmgdk::glm_kernel<T, V, 32, 8>, V, 32, 8, bmgdk::glm_max_threads<T, V, 8>()},
-    };
-    static const GlmVariant narrow[] = {
-        {bmgdk::glm_kernel<T, 1, 32, 1>, 1, 32, 1, bmgdk::glm_max_threads<T, 1, 1>()}, {bmgdk::glm_kernel<T, 1, 32, 2>, 1, 32, 2, bmgdk::glm_max_threads<T, 1, 2>()},
-        {bmgdk::glm_kernel<T, 1, 32, 4>, 1, 32, 4, bmgdk::glm_max_threads<T, 1, 4>()}, {bmgdk::glm_kernel<T, 1, 32, 8>, 1, 32, 8, bmgdk::glm_max_threads<T, 1, 8>()},
-    };
+#define BMGD_VAR(VEC, LPR, KCH) {bmgdk::glm_kernel<T, VEC, LPR, KCH, LG>, VEC, LPR, KCH, bmgdk::glm_max_threads<T, VEC, KCH>()}
+    static const GlmVariant wide[] = {BMGD_VAR(V, 8, 1), BMGD_VAR(V, 8, 2), BMGD_VAR(V, 8, 4),
+                                      BMGD_VAR(V, 8, 8), BMGD_VAR(V, 16, 8), BMGD_VAR(V, 32, 8)};
+    static const GlmVariant narrow[] = {BMGD_VAR(1, 32, 1), BMGD_VAR(1, 32, 2), BMGD_VAR(1, 32, 4), BMGD_VAR(1, 32, 8)};
+#undef BMGD_VAR
     if (aligned16) { *count = 6; return wide; }
     *count = 4;
     return narrow;
 }
 
-const GlmVariant* pick_variant(int dtype, int p, bool aligned16) {
+const GlmVariant* pick_variant(int dtype, int loss, int p, bool aligned16) {
     int cnt = 0;
-    const GlmVariant* v = dtype == BMGD_F64 ? glm_variants<double>(aligned16, &cnt) : glm_variants<float>(aligned16, &cnt);
+    const bool lg = loss == BMGD_LOSS_LOGISTIC;
+    const GlmVariant* v = dtype == BMGD_F64
+        ? (lg ? glm_variants<double, true>(aligned16, &cnt) : glm_variants<double, false>(aligned16, &cnt))
+        : (lg ? glm_variants<float, true>(aligned16, &cnt) : glm_variants<float, false>(aligned16, &cnt));
     for (int i = 0; i < cnt; ++i)
         if (v[i].cap() >= p) return &v[i];
     return nullptr;
@@ -190,7 +189,7 @@ int floor_pow2(int v) {
 }
 
 struct LaunchShape {
-    int S, cpc, nteams, threads, depth, passes, rb, pitch, smem;
+    int S, cpc, nteams, threads, depth, passes, rb, smem;
 };
 
 int max_active_clusters(bmgd* h, GlmKernel fn, int S, int threads, int smem, int* out) {
@@ -218,7 +217,8 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
                                   : ((c.Rc > 1 && var->max_threads() >= 512) ? 512 : 256);
     const int warps = L.threads / 32;
     const int spp = warps * gpw;  // rows a CTA works on at once (one sub-pass)
-    L.pitch = (int)align_up((int64_t)c.p * eb, 16);
+    const bool pre = var->kch * var->vec <= 16;
+    const int pitch = pcap * eb + 16;
 
     // cluster size
     int S = c.cluster_size;
@@ -232,9 +232,9 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
 
     // How many clusters can be resident depends on shared memory, which depends on the ring; ask with
     // the largest ring we would use (a smaller one can only admit more).
-    const int fixed_smem = bmgdk::glm_smem_plan(warps, gpw, 1, 0, L.pitch, pcap, eb, S).total_bytes;
+    const int fixed_smem = bmgdk::glm_smem_plan(warps, gpw, pre, 1, 0, pcap, eb, S).total_bytes;
     const int ring_budget = std::min(h->smem_optin - fixed_smem, 160 * 1024);
-    if (ring_budget < spp * (L.pitch + 16)) return BMGD_ERR_UNIMPLEMENTED;
+    if (ring_budget < spp * pitch) return BMGD_ERR_UNIMPLEMENTED;
     const int probe_smem = fixed_smem + ring_budget;
     BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn, cudaFuncAttributeMaxDynamicSharedMemorySize, probe_smem));
     if (S > 8) BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
@@ -267,21 +267,20 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     const int subpasses = std::max(1, (rows_per_cta + spp - 1) / spp);
 
     // sub-passes per ring stage: fewer, larger stages amortise the per-stage bookkeeping
-    const int subpass_bytes = spp * (L.pitch + 16);
+    const int subpass_bytes = spp * pitch;
     int rb = c.subpasses_per_stage ? c.subpasses_per_stage : var->lpr;
     rb = std::min(rb, var->lpr);
     rb = floor_pow2(std::max(1, std::min(rb, subpasses)));
-    const int stage_cap = c.subpasses_per_stage ? ring_budget / 2 : std::min(ring_budget / 3, 56 * 1024);
+    const int stage_cap = c.subpasses_per_stage ? ring_budget / 2 : std::min(ring_budget / 4, 40 * 1024);
     while (rb > 1 && rb * subpass_bytes > stage_cap) rb /= 2;
     L.rb = rb;
     L.passes = (subpasses + rb - 1) / rb;
     const int stage_bytes = rb * subpass_bytes;
-    int depth = c.pipeline_depth ? c.pipeline_depth : std::max(2, (128 * 1024) / stage_bytes);
-    depth = std::min(depth, 16);
-    while (depth > 1 && depth * stage_bytes > ring_budget) --depth;
+    int depth = c.pipeline_depth ? c.pipeline_depth : 4;  // the kernel keeps 2, 3 or 4 stages in flight
+    while (depth > 2 && depth * stage_bytes > ring_budget) --depth;
     if (depth * stage_bytes > ring_budget) return BMGD_ERR_UNIMPLEMENTED;
     L.depth = depth;
-    L.smem = bmgdk::glm_smem_plan(warps, gpw, rb, depth, L.pitch, pcap, eb, S).total_bytes;
+    L.smem = bmgdk::glm_smem_plan(warps, gpw, pre, rb, depth, pcap, eb, S).total_bytes;
     (void)rows;
     *out = L;
     return BMGD_OK;
@@ -324,7 +323,7 @@ int check_status_word(bmgd* h) {
 int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, int n, double lr, uint64_t seed) {
     const bmgd_config& c = h->cfg;
     const bool aligned16 = ((int64_t)c.p * h->tb) % 16 == 0 && ((uintptr_t)dx % 16) == 0;
-    const GlmVariant* var = pick_variant(c.dtype, c.p, aligned16);
+    const GlmVariant* var = pick_variant(c.dtype, c.loss, c.p, aligned16);
     if (!var) return BMGD_ERR_UNIMPLEMENTED;
     if (((uintptr_t)dx % h->tb) != 0 || ((uintptr_t)dy % h->tb) != 0) return BMGD_ERR_ARG;
     LaunchShape L{};
@@ -334,7 +333,7 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
     const uint32_t M = (uint32_t)((rows + n - 1) / n);
     const int chains_per_team = (c.Rc + L.nteams - 1) / L.nteams;
     const uint64_t steps_per_team = (uint64_t)chains_per_team * (uint64_t)rounds * M;
-    if (steps_per_team >= 0xFFFFFFF0ull) return BMGD_ERR_ARG;
+    if (steps_per_team * (uint64_t)L.passes >= 0xFFFFFFF0ull) return BMGD_ERR_ARG;
     if (h->tag_base + steps_per_team >= 0xFFFFFFF0ull) {
         // tags would wrap: wipe the packet area (on-stream, after earlier launches) and start over
         BMGD_CUDA(h, cudaMemsetAsync(h->base + h->lay.ll, 0, (size_t)(h->lay.status - h->lay.ll), h->compute));
@@ -348,10 +347,11 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
     P.status = reinterpret_cast<int*>(h->base + h->lay.status);
     P.seed = seed;
     P.timeout_ns = h->timeout_ns;
-    P.alpha = lr;
+    P.scale_full = lr / (double)n;
+    P.scale_last = lr / (double)(rows - (int64_t)(M - 1) * n);
     P.N0 = (uint32_t)rows; P.n = (uint32_t)n; P.M = M; P.T = rounds; P.p = c.p;
-    P.loss = c.loss; P.Rc = c.Rc; P.S = L.S; P.cpc = L.cpc; P.nteams = L.nteams;
-    P.passes = L.passes; P.rb = L.rb; P.depth = L.depth; P.pitch = L.pitch;
+    P.Rc = c.Rc; P.S = L.S; P.cpc = L.cpc; P.nteams = L.nteams;
+    P.passes = L.passes; P.rb = L.rb; P.depth = L.depth;
     P.q_full = (uint32_t)n / (uint32_t)(L.cpc * L.S); P.r_full = (uint32_t)n % (uint32_t)(L.cpc * L.S);
     P.ll_stride = c.p * 2;
     P.tag_base = (uint32_t)h->tag_base;
@@ -751,7 +751,7 @@ int bmgd_run_rounds_noalloc(const void* dev_x, const void* dev_y, int64_t rows, 
     const int tb = tmp.tb;
     if (((uintptr_t)dev_x % tb) != 0 || ((uintptr_t)dev_y % tb) != 0 || ((uintptr_t)dev_theta % tb) != 0) return BMGD_ERR_ARG;
     const bool aligned16 = ((int64_t)p * tb) % 16 == 0 && ((uintptr_t)dev_x % 16) == 0;
-    const GlmVariant* var = pick_variant(dtype, p, aligned16);
+    const GlmVariant* var = pick_variant(dtype, loss, p, aligned16);
     if (!var) return BMGD_ERR_UNIMPLEMENTED;
     LaunchShape L{};
     rc = plan_glm(&tmp, var, rows, n, &L);
@@ -759,7 +759,7 @@ int bmgd_run_rounds_noalloc(const void* dev_x, const void* dev_y, int64_t rows, 
 
     const uint32_t M = (uint32_t)((rows + n - 1) / n);
     const int chains_per_team = (Rc + L.nteams - 1) / L.nteams;
-    if ((uint64_t)chains_per_team * (uint64_t)rounds * M >= 0xFFFFFFF0ull) return BMGD_ERR_ARG;
+    if ((uint64_t)chains_per_team * (uint64_t)rounds * M * (uint64_t)L.passes >= 0xFFFFFFF0ull) return BMGD_ERR_ARG;
     if ((int64_t)L.nteams * L.cpc > kMaxClustersForExchange) return BMGD_ERR_LAUNCH;
     const size_t packet_bytes = (size_t)2 * kMaxClustersForExchange * p * 2 * 8;
     if (256 + packet_bytes > (size_t)BMGD_NOALLOC_SCRATCH_BYTES) return BMGD_ERR_CAPACITY;
@@ -776,10 +776,11 @@ int bmgd_run_rounds_noalloc(const void* dev_x, const void* dev_y, int64_t rows, 
     P.ll = reinterpret_cast<unsigned long long*>(scratch + 256);
     P.seed = seed;
     P.timeout_ns = 2000000000ull;
-    P.alpha = lr;
+    P.scale_full = lr / (double)n;
+    P.scale_last = lr / (double)(rows - (int64_t)(M - 1) * n);
     P.N0 = (uint32_t)rows; P.n = (uint32_t)n; P.M = M; P.T = rounds; P.p = p;
-    P.loss = loss; P.Rc = Rc; P.S = L.S; P.cpc = L.cpc; P.nteams = L.nteams;
-    P.passes = L.passes; P.rb = L.rb; P.depth = L.depth; P.pitch = L.pitch;
+    P.Rc = Rc; P.S = L.S; P.cpc = L.cpc; P.nteams = L.nteams;
+    P.passes = L.passes; P.rb = L.rb; P.depth = L.depth;
     P.q_full = (uint32_t)n / (uint32_t)(L.cpc * L.S); P.r_full = (uint32_t)n % (uint32_t)(L.cpc * L.S);
     P.ll_stride = p * 2;
     P.tag_base = 0;

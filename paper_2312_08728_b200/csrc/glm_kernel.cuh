@@ -13,10 +13,13 @@
 //   2. a group of LPR lanes owns one row: x.theta by an LPR-lane butterfly, the residual
 //      (x.theta - y, or sigmoid(x.theta) - y), then g += r * x with x still in registers, so a
 //      row is read from HBM once and from shared memory once;
-//   3. the group partials are summed in fixed order in shared memory, then across the cluster
-//      through distributed shared memory (every CTA pushes its partial to every peer), then
-//      across clusters through tagged 8-byte packets in global memory (value and step tag
-//      travel in one 64-bit store, so a reader needs no separate flag or fence);
+//   3. the group partials are summed in fixed order (shuffles, then shared memory).  With one
+//      cluster per chain every CTA pushes its partial to every peer through distributed shared
+//      memory and one cluster barrier follows.  With several clusters the partials are
+//      reduce-scattered inside the cluster (CTA r owns a slice of the predictors), the slice sums
+//      cross clusters as tagged 8-byte packets in global memory (value and step tag travel in one
+//      64-bit store, so a reader needs no separate flag or fence; only the slice owner polls), and
+//      the totals are pushed back to every peer before a second cluster barrier;
 //   4. every CTA applies theta <- theta - (alpha/n_m) g to its own register copy of theta.
 // All sums have a fixed order, so all CTAs hold bit-identical theta and runs are reproducible.
 //
@@ -42,22 +45,21 @@ struct GlmParams {
     int* status;          // [0] first error code, [1] abort flag
     unsigned long long seed;
     unsigned long long timeout_ns;
-    double alpha;
+    double scale_full;    // alpha / n: step size over a full mini-batch
+    double scale_last;    // alpha / (size of the ragged last mini-batch of a round)
     uint32_t N0;
     uint32_t n;           // mini-batch size
     uint32_t M;           // mini-batches per round
     int T;                // rounds
     int p;
-    int loss;             // 0 linear, 1 logistic
     int Rc;
     int S;                // cluster size
     int cpc;              // clusters per chain
     int nteams;
     int passes;           // ring stages per step
     int rb;               // sub-passes per ring stage (a power of two, at most LPR)
-    int depth;            // ring stages in flight
+    int depth;            // ring stages in flight: 2, 3 or 4
     uint32_t q_full, r_full;  // n / G and n % G: how a full mini-batch is dealt to the G CTAs
-    int pitch;            // bytes between rows in the ring (multiple of 16)
     int ll_stride;        // packets per cluster slot
     uint32_t tag_base;
     int fixed_partition;
@@ -75,24 +77,32 @@ __device__ __forceinline__ void cp_async(uint32_t dst_smem, const void* src) {
         asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst_smem), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_pending(int n) {
-    switch (n) {  // the operand must be an immediate
-        case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
-        case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
-        case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
-        case 3: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
-        case 4: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
-        case 5: asm volatile("cp.async.wait_group 5;" ::: "memory"); break;
-        case 6: asm volatile("cp.async.wait_group 6;" ::: "memory"); break;
-        case 7: asm volatile("cp.async.wait_group 7;" ::: "memory"); break;
-        case 8: asm volatile("cp.async.wait_group 8;" ::: "memory"); break;
-        case 9: asm volatile("cp.async.wait_group 9;" ::: "memory"); break;
-        case 10: asm volatile("cp.async.wait_group 10;" ::: "memory"); break;
-        case 11: asm volatile("cp.async.wait_group 11;" ::: "memory"); break;
-        case 12: asm volatile("cp.async.wait_group 12;" ::: "memory"); break;
-        case 13: asm volatile("cp.async.wait_group 13;" ::: "memory"); break;
-        case 14: asm volatile("cp.async.wait_group 14;" ::: "memory"); break;
-        default: asm volatile("cp.async.wait_group 15;" ::: "memory"); break;
+// cp.async.wait_group takes an immediate: the ring is 2, 3 or 4 stages deep.
+__device__ __forceinline__ void cp_async_wait_ring(int depth) {
+    if (depth == 4) asm volatile("cp.async.wait_group 3;" ::: "memory");
+    else if (depth == 3) asm volatile("cp.async.wait_group 2;" ::: "memory");
+    else asm volatile("cp.async.wait_group 1;" ::: "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
+// One predicated copy chunk at a constant byte offset from both addresses.
+template <int BYTES, int OFF>
+__device__ __forceinline__ void cp_async_at(uint32_t dst_smem, const void* src, uint32_t pred) {
+    if constexpr (BYTES == 16)
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %2, 0;\n\t@p cp.async.cg.shared.global [%0+%3], [%1+%3], 16;\n\t}"
+                     ::"r"(dst_smem), "l"(src), "r"(pred), "n"(OFF) : "memory");
+    else if constexpr (BYTES == 8)
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %2, 0;\n\t@p cp.async.ca.shared.global [%0+%3], [%1+%3], 8;\n\t}"
+                     ::"r"(dst_smem), "l"(src), "r"(pred), "n"(OFF) : "memory");
+    else
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %2, 0;\n\t@p cp.async.ca.shared.global [%0+%3], [%1+%3], 4;\n\t}"
+                     ::"r"(dst_smem), "l"(src), "r"(pred), "n"(OFF) : "memory");
+}
+template <int BYTES, int STRIDE, int K, int KCH>
+__device__ __forceinline__ void cp_async_chunks(uint32_t dst_smem, const void* src, uint32_t kmask) {
+    if constexpr (K < KCH) {
+        cp_async_at<BYTES, K * STRIDE>(dst_smem, src, kmask & (1u << K));
+        cp_async_chunks<BYTES, STRIDE, K + 1, KCH>(dst_smem, src, kmask);
     }
 }
 
@@ -109,6 +119,9 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t cta)
 }
 __device__ __forceinline__ void st_cluster(uint32_t addr, float v) {
     asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void st_shared_zero16(uint32_t addr) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0) : "memory");
 }
 __device__ __forceinline__ void st_cluster(uint32_t addr, double v) {
     asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(addr), "d"(v) : "memory");
@@ -133,7 +146,7 @@ __device__ __forceinline__ unsigned long long global_ns() {
     return t;
 }
 
-__device__ __forceinline__ float sigmoid_of(float u) { return 1.0f / (1.0f + expf(-u)); }
+__device__ __forceinline__ float sigmoid_of(float u) { return __fdividef(1.0f, 1.0f + __expf(-u)); }
 __device__ __forceinline__ double sigmoid_of(double u) { return 1.0 / (1.0 + exp(-u)); }
 
 // 32-bit words of a value, for the tagged packets
@@ -157,19 +170,23 @@ template <> struct Words<double> {
 // ---------------------------------------------------------------- shared-memory plan (host and device agree on it)
 
 struct GlmSmemPlan {
-    int warp_stage_bytes;  // one warp's share of one ring stage: its rows, then its y values
+    int pitch;             // bytes from one ring row to the next: the full predictor capacity, then 16 bytes for y
+    int warp_stage_bytes;  // one warp's share of one ring stage
     int ring_bytes;
+    int gpart_rows;        // partial-gradient rows summed per CTA
     int gpart_off, cpart_off, gfin_off;
     int total_bytes;
 };
 
-__host__ __device__ inline GlmSmemPlan glm_smem_plan(int warps, int gpw, int rb, int depth, int pitch, int pcap,
+__host__ __device__ inline GlmSmemPlan glm_smem_plan(int warps, int gpw, bool prereduce, int rb, int depth, int pcap,
                                                      int elem_bytes, int S) {
     GlmSmemPlan s;
-    s.warp_stage_bytes = rb * gpw * (pitch + 16);
+    s.pitch = pcap * elem_bytes + 16;
+    s.warp_stage_bytes = rb * gpw * s.pitch;
     s.ring_bytes = warps * depth * s.warp_stage_bytes;
+    s.gpart_rows = prereduce ? warps : warps * gpw;
     s.gpart_off = s.ring_bytes;
-    s.cpart_off = s.gpart_off + warps * gpw * pcap * elem_bytes;
+    s.cpart_off = s.gpart_off + s.gpart_rows * pcap * elem_bytes;
     s.gfin_off = s.cpart_off + 2 * S * pcap * elem_bytes;
     s.total_bytes = s.gfin_off + pcap * elem_bytes;
     return s;
@@ -177,7 +194,7 @@ __host__ __device__ inline GlmSmemPlan glm_smem_plan(int warps, int gpw, int rb,
 
 #ifdef BMGD_TRACE
 // Debug build only: clock stamps of CTA 0 at the phase boundaries of its first steps.
-constexpr int kTraceSteps = 64, kTracePhases = 8;
+constexpr int kTraceSteps = 64, kTracePhases = 16;
 __device__ long long g_trace[kTraceSteps * kTracePhases];
 #define BMGD_STAMP(ph)                                                                              \
     do {                                                                                            \
@@ -195,13 +212,19 @@ template <typename T, int VEC, int KCH>
 __host__ __device__ constexpr int glm_max_threads() {
     return (sizeof(T) == 8 || KCH * VEC >= 32) ? 256 : 512;
 }
+// Few values per lane: fold the row groups of a warp together by shuffles before shared memory.
+template <int VEC, int KCH>
+__host__ __device__ constexpr bool glm_prereduce() {
+    return KCH * VEC <= 16;
+}
 
 // How mini-batch rows [lo, lo+nm) are dealt to CTA g of G: a contiguous run of `cnt` rows from lo+a.
+// nsp is the number of sub-passes of the step in which the calling warp has at least one row.
 struct RowShare {
-    uint32_t lo, a, cnt;
+    uint32_t lo, a, cnt, nsp;
 };
 __device__ __forceinline__ RowShare row_share(uint32_t m, uint32_t n, uint32_t N0, uint32_t g, uint32_t G,
-                                              uint32_t q_full, uint32_t r_full) {
+                                              uint32_t q_full, uint32_t r_full, uint32_t warp_first, int spp_log2) {
     RowShare s;
     s.lo = m * n;
     const uint32_t nm = min(n, N0 - s.lo);
@@ -209,16 +232,75 @@ __device__ __forceinline__ RowShare row_share(uint32_t m, uint32_t n, uint32_t N
     if (nm != n) { q = nm / G; r = nm % G; }
     s.a = g * q + min(g, r);
     s.cnt = q + (g < r ? 1u : 0u);
+    s.nsp = (s.cnt > warp_first) ? ((s.cnt - warp_first - 1u) >> spp_log2) + 1u : 0u;
     return s;
+}
+
+// Sum `rows` values spaced `stride` elements apart, eight loads in flight at a time, fixed order.
+template <typename T>
+__device__ __forceinline__ T strided_sum(const T* col, int rows, int stride) {
+    T s0 = T(0), s1 = T(0);
+    for (int r0 = 0; r0 < rows; r0 += 8) {
+        T v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = (r0 + j < rows) ? col[(r0 + j) * stride] : T(0);
+        s0 += (v[0] + v[1]) + (v[2] + v[3]);
+        s1 += (v[4] + v[5]) + (v[6] + v[7]);
+    }
+    return s0 + s1;
+}
+
+// One row per LPR-lane group: residual from the dot product with theta, then g += r * x.
+// `rowp` is this lane's first chunk of the row in shared memory; y sits y_rel bytes from it.
+template <typename T, int VEC, int LPR, int KCH, bool LOGISTIC>
+__device__ __forceinline__ void row_step(const unsigned char* rowp, int y_rel, const T (&th)[KCH * VEC],
+                                         T (&gacc)[KCH * VEC]) {
+    constexpr int NV = KCH * VEC;
+    constexpr int CB = VEC * (int)sizeof(T);
+    T x[NV];
+#pragma unroll
+    for (int k = 0; k < KCH; ++k) {
+        if constexpr (CB == 16 && sizeof(T) == 4) {
+            const float4 v = *reinterpret_cast<const float4*>(rowp + k * LPR * CB);
+            x[k * VEC + 0] = v.x; x[k * VEC + 1] = v.y; x[k * VEC + 2] = v.z; x[k * VEC + 3] = v.w;
+        } else if constexpr (CB == 16) {
+            const double2 d = *reinterpret_cast<const double2*>(rowp + k * LPR * CB);
+            x[k * VEC + 0] = d.x; x[k * VEC + 1] = d.y;
+        } else {
+            x[k] = *reinterpret_cast<const T*>(rowp + k * LPR * CB);
+        }
+    }
+    const T yv = *reinterpret_cast<const T*>(rowp + y_rel);
+    T part[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) part[e] = T(0);
+#pragma unroll
+    for (int k = 0; k < KCH; ++k)
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) part[e] = fma(x[k * VEC + e], th[k * VEC + e], part[e]);
+    T dot = part[0];
+#pragma unroll
+    for (int e = 1; e < VEC; ++e) dot += part[e];
+#pragma unroll
+    for (int off = LPR / 2; off > 0; off >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, off);
+    // an empty slot has x = 0 and y = 0: whatever the residual is, it multiplies zeros
+    T res;
+    if constexpr (LOGISTIC) res = sigmoid_of(dot) - yv;
+    else res = dot - yv;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) gacc[i] = fma(res, x[i], gacc[i]);
 }
 
 // T: float or double.  VEC: elements per copy chunk (16 bytes worth, or 1 when rows are not
 // 16-byte multiples).  LPR: lanes per row.  KCH: chunks per lane.  A row has at most
-// LPR*KCH*VEC predictors.
+// PCAP = LPR*KCH*VEC predictors.  LOGISTIC: sigmoid residual instead of the linear one.
 //
 // Row slots of a CTA within one step are numbered u = (sp*W + warp)*GPW + grp, sp = sub-pass:
 // in sub-pass sp every warp works on GPW rows at once.  A ring stage holds `rb` sub-passes.
-template <typename T, int VEC, int LPR, int KCH>
+// A ring row is PCAP values wide whatever p is; the part beyond p is zeroed once and never written,
+// and a slot without a row is zero-filled, so the inner loop carries no predicates.
+// blockDim.x is 256, 512 or 1024.
+template <typename T, int VEC, int LPR, int KCH, bool LOGISTIC>
 __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(const GlmParams P) {
     constexpr int GPW = 32 / LPR;            // row groups per warp
     constexpr int NV = KCH * VEC;            // values per lane
@@ -226,6 +308,8 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
     constexpr int FPT = (PCAP + 255) / 256;  // features per thread in the reductions (blockDim >= 256)
     constexpr int CB = VEC * (int)sizeof(T); // copy chunk bytes
     constexpr int NW = Words<T>::N;
+    constexpr bool PRE = glm_prereduce<VEC, KCH>();
+    constexpr int YOFF = PCAP * (int)sizeof(T);  // y sits behind the predictors of its row
     constexpr uint32_t kNoRow = 0xFFFFFFFFu;
 
     extern __shared__ __align__(16) unsigned char smem[];
@@ -240,24 +324,37 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
     const int g = kc * S + rank;
     const int p = P.p, nchunks = p / VEC;
     const uint32_t N0 = P.N0, n = P.n, M = P.M;
-    const int T_rounds = P.T, passes = P.passes, RB = P.rb, D = P.depth, pitch = P.pitch;
+    const int T_rounds = P.T, passes = P.passes, RB = P.rb, D = P.depth;
+    const int spp_log2 = 31 - __clz(W * GPW);          // rows per sub-pass is a power of two
+    const uint32_t warp_first = (uint32_t)(warp * GPW); // first row slot of this warp in sub-pass 0
 
-    const GlmSmemPlan plan = glm_smem_plan(W, GPW, RB, D, pitch, PCAP, (int)sizeof(T), S);
-    unsigned char* my_ring = smem + (size_t)warp * D * plan.warp_stage_bytes;
-    const int y_off = RB * GPW * pitch;  // y values follow the rows of a warp's stage
+    const GlmSmemPlan plan = glm_smem_plan(W, GPW, PRE, RB, D, PCAP, (int)sizeof(T), S);
+    const int pitch = plan.pitch;
+    unsigned char* my_ring = smem + warp * D * plan.warp_stage_bytes;
     T* gpart = reinterpret_cast<T*>(smem + plan.gpart_off);
     T* cpart = reinterpret_cast<T*>(smem + plan.cpart_off);
     T* gfin = reinterpret_cast<T*>(smem + plan.gfin_off);
+    const int lane_off = grp * pitch + sub * CB;  // this lane's first chunk inside a sub-pass of its warp
+    const int subpass_bytes = GPW * pitch;
+    const int y_rel = YOFF - sub * CB;
 
-    const unsigned char* Xb = static_cast<const unsigned char*>(P.X);
+    const unsigned char* Xb = static_cast<const unsigned char*>(P.X) + sub * CB;
     const T* yb = static_cast<const T*>(P.y);
-    const size_t row_bytes = (size_t)p * sizeof(T);
+    const uint32_t row_bytes = (uint32_t)p * (uint32_t)sizeof(T);
     const FeistelDomain dom = make_domain(N0);
+    const int slice = (p + S - 1) / S;  // predictors owned by one CTA of a cluster in the sliced exchange
+    uint32_t kmask = 0;                 // chunk k of this lane lies inside the row
+#pragma unroll
+    for (int k = 0; k < KCH; ++k) kmask |= (sub + k * LPR < nchunks) ? (1u << k) : 0u;
+    const T scale_full = (T)P.scale_full, scale_last = (T)P.scale_last;
 
     const int nch = (team < P.Rc) ? (P.Rc - team + P.nteams - 1) / P.nteams : 0;
-    const long long nstages = (long long)nch * T_rounds * M * passes;
+    uint32_t to_issue = (uint32_t)nch * (uint32_t)T_rounds * M * (uint32_t)passes;  // the host keeps this below 2^32
 
-    if (S > 1) {  // peers must be running before anyone writes into their shared memory
+    // zero all of shared memory once: row tails beyond p and never-written slots must read as zero
+    for (int i = tid * 16; i < plan.total_bytes; i += nthreads * 16) st_shared_zero16(smem_u32(smem + i));
+    __syncthreads();
+    if (S > 1) {  // peers must be running (and zeroed) before anyone writes into their shared memory
         cluster_arrive_release();
         cluster_wait_acquire();
     }
@@ -266,31 +363,34 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
     int pf_ci = 0, pf_t = 0, pf_sidx = 0, pf_slot = 0;
     uint32_t pf_m = 0;
     uint32_t pf_rows = kNoRow;  // this lane's row of the current batch of 32 row slots
-    long long issued = 0;
     RoundKeys pfk = round_keys(P.seed, (uint32_t)team, 0u);
-    RowShare pfs = row_share(0u, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full);
+    RowShare pfs = row_share(0u, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full, warp_first, spp_log2);
 
     auto issue_one = [&]() {
-        if (issued < nstages) {
-            unsigned char* stage = my_ring + (size_t)pf_slot * plan.warp_stage_bytes;
-            for (int r = 0; r < RB; ++r) {
-                const int sp = pf_sidx * RB + r;
+        if (to_issue != 0u) {
+            --to_issue;
+            uint32_t dst = smem_u32(my_ring + pf_slot * plan.warp_stage_bytes) + lane_off;
+            int sp = pf_sidx * RB;
+            for (int r = 0; r < RB; ++r, ++sp, dst += subpass_bytes) {
                 const int bi = sp & (LPR - 1);
                 if (bi == 0) {  // a new batch: lane l takes sub-pass sp + l/GPW, group l%GPW
-                    const uint32_t u = ((uint32_t)(sp + lane / GPW) * (uint32_t)W + (uint32_t)warp) * GPW + (lane % GPW);
+                    const uint32_t u = (((uint32_t)(sp + lane / GPW)) << spp_log2) + warp_first + (lane % GPW);
                     pf_rows = (u < pfs.cnt) ? perm_index(pfs.lo + pfs.a + u, dom, pfk) : kNoRow;
                 }
-                const uint32_t row = __shfl_sync(0xFFFFFFFFu, pf_rows, bi * GPW + grp);
-                if (row != kNoRow) {
-                    const unsigned char* src = Xb + (size_t)row * row_bytes;
-                    const int slot_row = r * GPW + grp;
-                    const uint32_t dst = smem_u32(stage + slot_row * pitch);
+                if ((uint32_t)sp < pfs.nsp) {  // otherwise the whole warp skips this sub-pass, here and in the compute loop
+                    const uint32_t row = __shfl_sync(0xFFFFFFFFu, pf_rows, bi * GPW + grp);
+                    if (row != kNoRow) {
+                        cp_async_chunks<CB, LPR * CB, 0, KCH>(dst, Xb + (size_t)row * row_bytes, kmask);
+                        cp_async_at<(int)sizeof(T), 0>(dst + y_rel, yb + row, sub == 0 ? 1u : 0u);
+                    } else {  // no row for this slot: it must contribute nothing
 #pragma unroll
-                    for (int k = 0; k < KCH; ++k) {
-                        const int c = sub + k * LPR;
-                        if (c < nchunks) cp_async<CB>(dst + c * CB, src + (size_t)c * CB);
+                        for (int k = 0; k < KCH; ++k) {
+                            if constexpr (CB == 16) st_shared_zero16(dst + k * LPR * CB);
+                            else if constexpr (CB == 8) asm volatile("st.shared.b64 [%0], %1;" ::"r"(dst + k * LPR * CB), "l"(0ull) : "memory");
+                            else asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst + k * LPR * CB), "r"(0) : "memory");
+                        }
+                        if (sub == 0) st_shared_zero16(dst + y_rel);
                     }
-                    if (sub == 0) cp_async<(int)sizeof(T)>(smem_u32(stage + y_off + slot_row * 16), yb + row);
                 }
             }
             if (++pf_sidx == passes) {
@@ -302,12 +402,11 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                         pfk = round_keys(P.seed, (uint32_t)(team + pf_ci * P.nteams),
                                          P.fixed_partition ? 0u : (uint32_t)pf_t);
                 }
-                pfs = row_share(pf_m, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full);
+                pfs = row_share(pf_m, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full, warp_first, spp_log2);
             }
             if (++pf_slot == D) pf_slot = 0;
         }
         cp_async_commit();
-        ++issued;
         __syncwarp();  // lanes walked the cycle for different lengths: meet again before any aligned barrier
     };
 
@@ -316,7 +415,6 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
     int cs_slot = 0;         // ring slot the compute cursor reads next
     uint32_t step_count = 0; // steps this team has finished in this launch
     bool aborted = false;
-    const bool logistic = (P.loss == 1);
 
     for (int ci = 0; ci < nch; ++ci) {
         const int chain = team + ci * P.nteams;
@@ -332,66 +430,26 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
 
         for (int t = 0; t < T_rounds; ++t) {
             for (uint32_t m = 0; m < M; ++m) {
-                const RowShare sh = row_share(m, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full);
-                const uint32_t nm = min(n, N0 - sh.lo);
+                const RowShare sh = row_share(m, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full, warp_first, spp_log2);
                 BMGD_STAMP(0);
 
                 T gacc[NV];
 #pragma unroll
                 for (int i = 0; i < NV; ++i) gacc[i] = T(0);
 
+                int sp_left = (int)sh.nsp;  // sub-passes of this step in which the warp still has rows
                 for (int sidx = 0; sidx < passes; ++sidx) {
-                    cp_async_wait_pending(D - 1);
+                    cp_async_wait_ring(D);
                     __syncwarp();
-                    const unsigned char* stage = my_ring + (size_t)cs_slot * plan.warp_stage_bytes;
+                    const unsigned char* rowp = my_ring + cs_slot * plan.warp_stage_bytes + lane_off;
                     if (++cs_slot == D) cs_slot = 0;
-
-                    for (int r = 0; r < RB; ++r) {
-                        const uint32_t u = ((uint32_t)(sidx * RB + r) * (uint32_t)W + (uint32_t)warp) * GPW + grp;
-                        const bool valid = u < sh.cnt;
-                        const int slot_row = r * GPW + grp;
-
-                        T x[NV];
-                        const unsigned char* rowp = stage + slot_row * pitch;
-#pragma unroll
-                        for (int k = 0; k < KCH; ++k) {
-                            const int c = sub + k * LPR;
-                            if (valid && c < nchunks) {
-                                if constexpr (CB == 16 && sizeof(T) == 4) {
-                                    const float4 v = *reinterpret_cast<const float4*>(rowp + c * 16);
-                                    x[k * VEC + 0] = v.x; x[k * VEC + 1] = v.y; x[k * VEC + 2] = v.z; x[k * VEC + 3] = v.w;
-                                } else if constexpr (CB == 16) {
-                                    const double2 d = *reinterpret_cast<const double2*>(rowp + c * 16);
-                                    x[k * VEC + 0] = d.x; x[k * VEC + 1] = d.y;
-                                } else {
-                                    x[k] = *reinterpret_cast<const T*>(rowp + c * CB);
-                                }
-                            } else {
-#pragma unroll
-                                for (int e = 0; e < VEC; ++e) x[k * VEC + e] = T(0);
-                            }
-                        }
-                        T part[VEC];
-#pragma unroll
-                        for (int e = 0; e < VEC; ++e) part[e] = T(0);
-#pragma unroll
-                        for (int k = 0; k < KCH; ++k)
-#pragma unroll
-                            for (int e = 0; e < VEC; ++e) part[e] = fma(x[k * VEC + e], th[k * VEC + e], part[e]);
-                        T dot = part[0];
-#pragma unroll
-                        for (int e = 1; e < VEC; ++e) dot += part[e];
-#pragma unroll
-                        for (int off = LPR / 2; off > 0; off >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, off);
-
-                        T res = T(0);
-                        if (valid) {
-                            const T yv = *reinterpret_cast<const T*>(stage + y_off + slot_row * 16);
-                            res = (logistic ? sigmoid_of(dot) : dot) - yv;
-                        }
-#pragma unroll
-                        for (int i = 0; i < NV; ++i) gacc[i] = fma(res, x[i], gacc[i]);
+                    int nsub = min(sp_left, RB);
+                    sp_left -= nsub;
+                    for (; nsub >= 2; nsub -= 2, rowp += 2 * subpass_bytes) {  // two independent rows in flight per group
+                        row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, y_rel, th, gacc);
+                        row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + subpass_bytes, y_rel, th, gacc);
                     }
+                    if (nsub) row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, y_rel, th, gacc);
                     if (sidx + 1 < passes) {  // refill the slot just read; the last one of a step waits for a barrier
                         __syncwarp();
                         issue_one();
@@ -399,14 +457,24 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                 }
                 BMGD_STAMP(1);
 
-                // ---- sum the group partials of this CTA in fixed order
-                {
-                    T* gp = gpart + (size_t)(warp * GPW + grp) * PCAP;
+                // ---- sum the partial gradients of this CTA in fixed order
+                if constexpr (PRE) {
+#pragma unroll
+                    for (int off = LPR; off < 32; off <<= 1)
+#pragma unroll
+                        for (int i = 0; i < NV; ++i) gacc[i] += __shfl_xor_sync(0xFFFFFFFFu, gacc[i], off);
+                }
+                if (!PRE || grp == 0) {
+                    T* gp = gpart + (PRE ? warp : warp * GPW + grp) * PCAP + sub * VEC;
 #pragma unroll
                     for (int k = 0; k < KCH; ++k) {
-                        const int c = sub + k * LPR;
-#pragma unroll
-                        for (int e = 0; e < VEC; ++e) gp[c * VEC + e] = gacc[k * VEC + e];
+                        if constexpr (CB == 16 && sizeof(T) == 4)
+                            *reinterpret_cast<float4*>(gp + k * LPR * VEC) =
+                                make_float4(gacc[k * VEC], gacc[k * VEC + 1], gacc[k * VEC + 2], gacc[k * VEC + 3]);
+                        else if constexpr (CB == 16)
+                            *reinterpret_cast<double2*>(gp + k * LPR * VEC) = make_double2(gacc[k * VEC], gacc[k * VEC + 1]);
+                        else
+                            gp[k * LPR] = gacc[k];
                     }
                 }
                 if (S == 1 && cpc == 1) {
@@ -415,134 +483,157 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                 }
                 __syncthreads();
                 BMGD_STAMP(2);
-                const int spp = W * GPW;
                 T tot[FPT];
 #pragma unroll
                 for (int i = 0; i < FPT; ++i) {
                     const int f = tid + i * nthreads;
-                    T s0 = T(0), s1 = T(0), s2 = T(0), s3 = T(0);
-                    if (f < p) {
-                        const T* col = gpart + f;
-                        int r4 = 0;
-                        for (; r4 + 3 < spp; r4 += 4) {
-                            s0 += col[(size_t)(r4 + 0) * PCAP];
-                            s1 += col[(size_t)(r4 + 1) * PCAP];
-                            s2 += col[(size_t)(r4 + 2) * PCAP];
-                            s3 += col[(size_t)(r4 + 3) * PCAP];
-                        }
-                        for (; r4 < spp; ++r4) s0 += col[(size_t)r4 * PCAP];
-                    }
-                    tot[i] = (s0 + s1) + (s2 + s3);
+                    tot[i] = (f < p) ? strided_sum(gpart + f, plan.gpart_rows, PCAP) : T(0);
                 }
                 BMGD_STAMP(3);
 
                 const int parity = (int)(step_count & 1u);
+                T* cp = cpart + parity * S * PCAP;
 
-                // ---- across the cluster: push to every peer, one barrier, sum locally
-                if (S > 1) {
-                    T* cp = cpart + (size_t)parity * S * PCAP;
-                    const uint32_t mine = smem_u32(cp + (size_t)rank * PCAP);
+                if (cpc == 1) {
+                    // ---- one cluster per chain: push to every peer, one barrier, sum locally
+                    if (S > 1) {
+                        const uint32_t mine = smem_u32(cp + rank * PCAP);
+#pragma unroll
+                        for (int i = 0; i < FPT; ++i) {
+                            const int f = tid + i * nthreads;
+                            if (f < p)
+                                for (int peer = 0; peer < S; ++peer)
+                                    st_cluster(map_to_cta(mine + f * (uint32_t)sizeof(T), (uint32_t)peer), tot[i]);
+                        }
+                        __syncwarp();
+                        cluster_arrive_release();
+                        issue_one();  // the copies for a later stage go out while the barrier completes
+                        cluster_wait_acquire();
+#pragma unroll
+                        for (int i = 0; i < FPT; ++i) {
+                            const int f = tid + i * nthreads;
+                            tot[i] = (f < p) ? strided_sum(cp + f, S, PCAP) : T(0);
+                        }
+                    }
+                    BMGD_STAMP(4);
+                    BMGD_STAMP(5);
 #pragma unroll
                     for (int i = 0; i < FPT; ++i) {
                         const int f = tid + i * nthreads;
-                        if (f < p)
-                            for (int peer = 0; peer < S; ++peer)
-                                st_cluster(map_to_cta(mine + f * (uint32_t)sizeof(T), (uint32_t)peer), tot[i]);
+                        if (f < p) gfin[f] = tot[i];
                     }
-                    __syncwarp();
-                    cluster_arrive_release();
-                    issue_one();  // the copies for a later stage go out while the barrier completes
-                    cluster_wait_acquire();
+                    __syncthreads();
+                } else {
+                    // ---- several clusters per chain: reduce-scatter in the cluster, packets between the slice
+                    //      owners of different clusters, all-gather of the totals in the cluster
+                    if (S > 1) {
+                        const uint32_t mine = smem_u32(cp + rank * PCAP);
 #pragma unroll
-                    for (int i = 0; i < FPT; ++i) {
-                        const int f = tid + i * nthreads;
-                        T s = T(0);
-                        if (f < p)
-                            for (int r2 = 0; r2 < S; ++r2) s += cp[(size_t)r2 * PCAP + f];
-                        tot[i] = s;
+                        for (int i = 0; i < FPT; ++i) {
+                            const int f = tid + i * nthreads;
+                            if (f < p) st_cluster(map_to_cta(mine + f * (uint32_t)sizeof(T), (uint32_t)(f / slice)), tot[i]);
+                        }
+                        __syncwarp();
+                        cluster_arrive_release();
+                        issue_one();
+                        cluster_wait_acquire();
                     }
-                }
-                BMGD_STAMP(4);
-
-                // ---- across clusters: tagged packets through global memory
-                if (cpc > 1) {
+                    BMGD_STAMP(4);
                     const uint32_t tag = P.tag_base + step_count + 1u;
-                    unsigned long long* slot =
-                        P.ll + ((size_t)(team * 2 + parity) * cpc) * (size_t)P.ll_stride;
+                    unsigned long long* slot = P.ll + ((size_t)(team * 2 + parity) * cpc) * (size_t)P.ll_stride;
+                    // thread j of the CTA owns predictor f = rank*slice + j of the slice (all of them if S == 1)
 #pragma unroll
                     for (int i = 0; i < FPT; ++i) {
-                        const int f = tid + i * nthreads;
-                        if (f < p && (f % S) == rank) {
+                        const int j = tid + i * nthreads;
+                        const int f = rank * slice + j;
+                        if (j < slice && f < p) {
+                            const T mine_sum = (S > 1) ? strided_sum(cp + f, S, PCAP) : tot[i];
 #pragma unroll
                             for (int w = 0; w < NW; ++w)
                                 st_packet(slot + (size_t)kc * P.ll_stride + f * NW + w,
-                                          ((unsigned long long)tag << 32) | Words<T>::get(tot[i], w));
+                                          ((unsigned long long)tag << 32) | Words<T>::get(mine_sum, w));
                         }
                     }
                     if (S == 1) issue_one();
 #pragma unroll
                     for (int i = 0; i < FPT; ++i) {
-                        const int f = tid + i * nthreads;
-                        T s = T(0);
-                        if (f < p) {
-                            unsigned long long v[kMaxCpc][NW];
-                            unsigned long long t0 = 0;
-                            uint32_t spins = 0;
-                            while (!aborted) {
-                                bool ok = true;
+                        const int j = tid + i * nthreads;
+                        const int f = rank * slice + j;
+                        if (j >= slice || f >= p) continue;
+                        unsigned long long v[kMaxCpc][NW];
+                        unsigned long long t0 = 0;
+                        uint32_t spins = 0;
+                        while (!aborted) {
+                            bool ok = true;
 #pragma unroll
-                                for (int k = 0; k < kMaxCpc; ++k) {
-                                    if (k < cpc) {
+                            for (int k = 0; k < kMaxCpc; ++k) {
+                                if (k < cpc) {
 #pragma unroll
-                                        for (int w = 0; w < NW; ++w) {
-                                            v[k][w] = ld_packet(slot + (size_t)k * P.ll_stride + f * NW + w);
-                                            ok &= ((uint32_t)(v[k][w] >> 32) == tag);
-                                        }
-                                    }
-                                }
-                                if (ok) break;
-                                if ((++spins & 0x3FFu) == 0u) {
-                                    const unsigned long long now = global_ns();
-                                    if (t0 == 0) t0 = now;
-                                    if (now - t0 > P.timeout_ns || ((volatile int*)P.status)[1] != 0) {
-                                        atomicCAS(P.status, 0, kStatusTimeout);
-                                        atomicExch(P.status + 1, 1);
-                                        aborted = true;
+                                    for (int w = 0; w < NW; ++w) {
+                                        v[k][w] = ld_packet(slot + (size_t)k * P.ll_stride + f * NW + w);
+                                        ok &= ((uint32_t)(v[k][w] >> 32) == tag);
                                     }
                                 }
                             }
-                            if (!aborted) {
-#pragma unroll
-                                for (int k = 0; k < kMaxCpc; ++k) {
-                                    if (k < cpc) {
-                                        uint32_t w32[NW];
-#pragma unroll
-                                        for (int w = 0; w < NW; ++w) w32[w] = (uint32_t)v[k][w];
-                                        s += Words<T>::make(w32);
-                                    }
+                            if (ok) break;
+                            if ((++spins & 0x3FFu) == 0u) {
+                                const unsigned long long now = global_ns();
+                                if (t0 == 0) t0 = now;
+                                if (now - t0 > P.timeout_ns || ((volatile int*)P.status)[1] != 0) {
+                                    atomicCAS(P.status, 0, kStatusTimeout);
+                                    atomicExch(P.status + 1, 1);
+                                    aborted = true;
                                 }
                             }
                         }
-                        tot[i] = s;
+                        T s = T(0);
+                        if (!aborted) {
+#pragma unroll
+                            for (int k = 0; k < kMaxCpc; ++k) {
+                                if (k < cpc) {
+                                    uint32_t w32[NW];
+#pragma unroll
+                                    for (int w = 0; w < NW; ++w) w32[w] = (uint32_t)v[k][w];
+                                    s += Words<T>::make(w32);
+                                }
+                            }
+                        }
+                        if (S > 1) {
+                            const uint32_t dst = smem_u32(gfin + f);
+                            for (int peer = 0; peer < S; ++peer) st_cluster(map_to_cta(dst, (uint32_t)peer), s);
+                        } else {
+                            gfin[f] = s;
+                        }
+                    }
+                    BMGD_STAMP(5);
+                    if (S > 1) {
+                        __syncwarp();
+                        cluster_arrive_release();
+                        cluster_wait_acquire();
+                    } else {
+                        __syncthreads();
                     }
                 }
-                BMGD_STAMP(5);
+                BMGD_STAMP(6);
 
                 // ---- everyone updates its own copy of theta
+                const T scale = (min(n, N0 - sh.lo) == n) ? scale_full : scale_last;
+                {
+                    const T* gf = gfin + sub * VEC;
 #pragma unroll
-                for (int i = 0; i < FPT; ++i) {
-                    const int f = tid + i * nthreads;
-                    if (f < PCAP) gfin[f] = (f < p) ? tot[i] : T(0);
-                }
-                // a thread that gave up tells the rest of its CTA, so that no one else waits out its own budget
-                aborted = __syncthreads_or(aborted ? 1 : 0) != 0;
-                BMGD_STAMP(6);
-                const T scale = (T)(P.alpha / (double)nm);
+                    for (int k = 0; k < KCH; ++k) {
+                        if constexpr (CB == 16 && sizeof(T) == 4) {
+                            const float4 v = *reinterpret_cast<const float4*>(gf + k * LPR * VEC);
+                            th[k * VEC + 0] = fma(-scale, v.x, th[k * VEC + 0]);
+                            th[k * VEC + 1] = fma(-scale, v.y, th[k * VEC + 1]);
+                            th[k * VEC + 2] = fma(-scale, v.z, th[k * VEC + 2]);
+                            th[k * VEC + 3] = fma(-scale, v.w, th[k * VEC + 3]);
+                        } else {
 #pragma unroll
-                for (int k = 0; k < KCH; ++k) {
-                    const int c = sub + k * LPR;
-#pragma unroll
-                    for (int e = 0; e < VEC; ++e) th[k * VEC + e] -= scale * gfin[c * VEC + e];
+                            for (int e = 0; e < VEC; ++e)
+                                th[k * VEC + e] = fma(-scale, gf[k * LPR * VEC + e], th[k * VEC + e]);
+                        }
+                    }
                 }
                 BMGD_STAMP(7);
                 ++step_count;
@@ -559,7 +650,7 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
             }
         }
     }
-    cp_async_wait_pending(0);
+    cp_async_wait_all();
 }
 
 // Writes out[j] = pi(j) for one (seed, chain, round): the shuffle exactly as the step kernel uses it.

@@ -68,7 +68,7 @@ SMALL = Workload("small", LOSS_LOGISTIC, DTYPE_F32, N=6_000, p=40, K=2, n=500, T
     dict(cluster_size=8, ctas_per_chain=64),
     dict(cluster_size=8, ctas_per_chain=8, threads_per_cta=512),
     dict(cluster_size=8, ctas_per_chain=16, pipeline_depth=2),
-    dict(cluster_size=8, ctas_per_chain=16, pipeline_depth=16),
+    dict(cluster_size=8, ctas_per_chain=16, pipeline_depth=3),
     dict(cluster_size=1, ctas_per_chain=1, subpasses_per_stage=1),
     dict(cluster_size=1, ctas_per_chain=1, subpasses_per_stage=4, pipeline_depth=3),
     dict(cluster_size=2, ctas_per_chain=2, subpasses_per_stage=8),
