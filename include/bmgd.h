@@ -60,7 +60,9 @@ enum {
     BMGD_FLAG_FIXED_PARTITION = 1u, /* reuse round 0's partition in every round: the fixed-partition
                                        assumption under which Eq. (3.1)-(3.3) are derived */
     BMGD_FLAG_NO_SLOTS = 2u,        /* allocate no buffer slots: only bmgd_run_rounds_resident is used */
-    BMGD_FLAG_TIMING = 4u           /* record CUDA events round every launch and copy (bmgd_get_stats) */
+    BMGD_FLAG_TIMING = 4u,          /* record CUDA events round every launch and copy (bmgd_get_stats) */
+    BMGD_FLAG_SOFTMAX_CUDA_CORES = 8u /* softmax: run the two contractions on the CUDA cores, not the tensor cores
+                                       (same bf16 inputs; for cross-checking the tensor-core path) */
 };
 
 /* Everything bmgd_create cannot say.  Fill with bmgd_config_init, then change fields. */

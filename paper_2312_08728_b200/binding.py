@@ -24,6 +24,7 @@ ERR_NONFINITE, ERR_LAUNCH, ERR_UNIMPLEMENTED, ERR_STATE = -6, -7, -8, -9
 FLAG_FIXED_PARTITION = 1
 FLAG_NO_SLOTS = 2
 FLAG_TIMING = 4
+FLAG_SOFTMAX_CUDA_CORES = 8
 
 # every symbol include/bmgd.h declares
 EXPORTS = (

@@ -427,7 +427,8 @@ int run_any(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
         int rc = bmgdk::softmax_run(dx, dy, rows, h->cfg.p, h->cfg.C, h->base + h->lay.theta,
                                    h->base + h->lay.softmax_scratch, reinterpret_cast<int*>(h->base + h->lay.status),
                                    rounds, n, lr, seed, (h->cfg.flags & BMGD_FLAG_FIXED_PARTITION) ? 1 : 0,
-                                   h->timeout_ns, h->cfg.cluster_size, h->cfg.threads_per_cta, h->cfg.pipeline_depth,
+                                   h->timeout_ns, h->cfg.cluster_size, h->cfg.threads_per_cta,
+                                   (h->cfg.flags & BMGD_FLAG_SOFTMAX_CUDA_CORES) ? 1 : 0,
                                    h->sm_count, h->smem_optin, h->compute, &info);
         if (rc != BMGD_OK) {
             if (info.cuda_error) h->last_cuda = info.cuda_error;

@@ -1,0 +1,95 @@
+"""Parity of the softmax step kernel (bf16 rows, fp32 W) with the CPU oracle, through the C ABI.
+
+Stated tolerance: relative L2 error of W at most 2e-2.  The oracle reads the same bf16 rows widened exactly
+and computes in fp64; the kernel rounds W and the residuals to bf16 for its two contractions.
+Both contraction paths are checked: tensor cores (default) and CUDA cores (same inputs, same layout).
+"""
+import numpy as np
+import pytest
+
+from paper_2312_08728_b200.inputs import WORKLOADS, Workload, LOSS_SOFTMAX, DTYPE_BF16
+
+from helpers import TOL, buffers_of, gpu_job, oracle_job, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+CUDA_CORES = 8  # BMGD_FLAG_SOFTMAX_CUDA_CORES
+
+
+def job(p, C=10, N=2_000, K=1, n=256, T=2, lr=0.1, epochs=1, seed=4):
+    return Workload(f"smx-p{p}", LOSS_SOFTMAX, DTYPE_BF16, N=N, p=p, K=K, n=n, T=T, lr=lr, epochs=epochs, C=C, seed=seed)
+
+
+def check(w, flags, mode="resident", tol=None):
+    bufs = buffers_of(w)
+    theta, stats = gpu_job(w, bufs, mode=mode, flags=flags)
+    want = oracle_job(w, bufs)[0]
+    err = rel_l2(theta[0], want)
+    assert err <= (tol or TOL[w.dtype]), (w.name, err, stats)
+    return theta[0], stats, err
+
+
+@pytest.mark.parametrize("p", [128, 192, 384, 1024, 3072])
+def test_cuda_core_path_matches_oracle(p):
+    """One CTA (p=128, 192), small clusters and the full 16-CTA cluster of the image-shaped workload."""
+    check(job(p), CUDA_CORES)
+
+
+@pytest.mark.parametrize("p", [128, 192, 384, 1024, 2048, 3072])
+def test_tensor_core_path_matches_oracle(p):
+    _, stats, _ = check(job(p), 0)
+    assert stats["cluster_size"] * stats["smem_bytes"] > 0
+
+
+def test_tensor_and_cuda_core_paths_agree_closely():
+    """Same bf16 inputs and fp32 accumulation: the two paths differ only in summation order."""
+    w = job(3072, N=1_500, T=1)
+    a, _, _ = check(w, 0)
+    b, _, _ = check(w, CUDA_CORES)
+    assert rel_l2(a, b) <= 1e-3
+
+
+@pytest.mark.parametrize("N,n,C", [(300, 256, 10), (256, 256, 2), (257, 128, 16), (40, 7, 3), (1, 1, 2)])
+def test_ragged_and_small_batches(N, n, C):
+    check(job(384, C=C, N=N, n=n, T=3, lr=0.05), 0)
+
+
+def test_two_class_softmax_follows_logistic_with_doubled_rate():
+    """The exact C = 2 identity, on the GPU: w_1 - w_0 of the softmax chain equals the fp32 logistic chain at 2*alpha
+    up to the bf16 rounding of the softmax path."""
+    import oracle
+    from paper_2312_08728_b200 import inputs
+    w = job(128, C=2, N=1_000, n=100, T=2, lr=0.05)
+    X, lab = inputs.make_buffer(w, 0)
+    theta, _ = gpu_job(w, [(X, lab)], mode="resident")
+    th = np.zeros(128)
+    oracle.run_rounds(oracle.LOGISTIC, X, lab.double(), th, w.T, w.n, 2 * w.lr, inputs.buffer_seed(w.seed, 0, 0, 1))
+    assert rel_l2(theta[0][:, 1] - theta[0][:, 0], th) <= 2e-2
+
+
+def test_slots_path_and_chaining_over_buffers():
+    w = job(3072, N=1_200, K=3, n=256, T=2, epochs=2)
+    check(w, 0, mode="slots")
+
+
+def test_cfg4_one_full_buffer():
+    """One full buffer of the image-shaped workload: 20,000 x 3,072 bf16, C=10, n=256 (last mini-batch 32 rows), T=4."""
+    w = WORKLOADS["cfg4"].scaled(N=20_000, K=1, epochs=1)
+    _, stats, err = check(w, 0)
+    assert stats["steps"] == 4 * 79
+
+
+def test_unsupported_shapes_are_refused_not_miscomputed():
+    from paper_2312_08728_b200.binding import BmgdError, ERR_UNIMPLEMENTED
+    for w in (job(100), job(384, n=300), job(128 * 17)):
+        with pytest.raises(BmgdError) as e:
+            gpu_job(w, buffers_of(w), mode="resident")
+        assert e.value.status == ERR_UNIMPLEMENTED
+
+
+def test_bitwise_reproducible():
+    w = job(1024, N=1_000, T=2)
+    bufs = buffers_of(w)
+    a, _ = gpu_job(w, bufs, mode="resident")
+    b, _ = gpu_job(w, bufs, mode="resident")
+    assert np.array_equal(a, b)
