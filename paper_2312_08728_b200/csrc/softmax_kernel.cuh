@@ -6,7 +6,7 @@
 // One thread-block cluster of S CTAs works on the chain, split by predictors: CTA r owns the slice
 // [r*ps, (r+1)*ps) of the p predictors (ps = NP panels of 64), i.e. ps rows of W.  Per step:
 //   1. the CTA's slice of the mini-batch rows (256 row slots x ps bf16) was gathered by cp.async into
-//      shared memory one step ahead, as NP panels of [256 rows][128 bytes] with the 128-byte swizzle
+//      shared memory one step ahead by sixteen producer warps, as NP panels of [256 rows][128 bytes] with the 128-byte swizzle
 //      the tensor core reads (16-byte chunk index XOR row%8);
 //   2. forward: partial logits Zp = X_slice W_slice, bf16 x bf16 -> fp32, on the 5th-generation
 //      tensor cores (tcgen05.mma, M=128 N=16 K=16, accumulator in tensor memory), A = the panels
@@ -31,7 +31,7 @@
 
 namespace bmgdk {
 
-constexpr int kSmxThreads = 384;
+constexpr int kSmxThreads = 768;     // 8 compute warps (one thread per row slot) + 16 producer warps
 constexpr int kSmxRows = 256;       // row slots per step (mini-batch size limit)
 constexpr int kSmxMaxPanels = 3;    // 64-predictor panels per CTA slice
 constexpr int kSmxClasses = 16;     // padded class count
@@ -86,6 +86,14 @@ __device__ __forceinline__ void st_cluster_v4(uint32_t addr, float a, float b, f
 }
 __device__ __forceinline__ void st_cluster_u16(uint32_t addr, unsigned short v) {
     asm volatile("st.shared::cluster.u16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
+}
+
+// named CTA barriers: `count` threads take part, by arriving (no wait) or by arriving and waiting
+__device__ __forceinline__ void named_arrive(int id, int count) {
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void named_sync(int id, int count) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
 // ---------------------------------------------------------------- mbarrier and proxy helpers
@@ -199,7 +207,6 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
     unsigned char* wt = smem + plan.wt_off;
     float* zpart = reinterpret_cast<float*>(smem + plan.zpart_off);
     unsigned char* rbuf = smem + plan.r_off;
-    uint32_t* idx = reinterpret_cast<uint32_t*>(smem + plan.idx_off);
     int* lab = reinterpret_cast<int*>(smem + plan.lab_off);
     const uint32_t mma_bar = smem_u32(smem + plan.bar_off);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + plan.bar_off + 16);
@@ -262,38 +269,49 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
         const int t = P.fixed_partition ? 0 : (int)(step / M);
         if (t != rk_round) { rk = round_keys(P.seed, 0u, (uint32_t)t); rk_round = t; }
     };
-    int next_label = -1;  // label of the row slot this thread will own in the next step
     auto gather = [&](uint32_t step, int b) {
-        // all threads; ends with a commit.  Row indices go through idx[b]; labels are fetched into a register.
+        // copies the step's 256 row slots (this CTA's NP*8 chunks of 16 bytes each) into the swizzled panels of
+        // buffer b and the owned labels into lab[b].  No barrier inside; ends with a commit by every thread.
         uint32_t lo, nm;
         step_rows(step, lo, nm);
         keys_for(step);
-        uint32_t my_row = 0xFFFFFFFFu;
-        if (tid < kSmxRows) {
-            if ((uint32_t)tid < nm) my_row = perm_index(lo + (uint32_t)tid, dom, rk);
-            idx[b * kSmxRows + tid] = my_row;
-        }
-        next_label = -1;
-        if (tid < RO) {
-            const uint32_t slot = (uint32_t)(rank * RO + tid);
-            if (slot < nm) next_label = P.y[perm_index(lo + slot, dom, rk)];
-        }
-        __syncthreads();
-        const int chunks_per_row = NP * 8;
-        const uint32_t dst0 = smem_u32(xbuf[b]);
-        for (int q = tid; q < kSmxRows * chunks_per_row; q += kSmxThreads) {
-            const int row = q / chunks_per_row, chunk = q % chunks_per_row;
-            const uint32_t r = idx[b * kSmxRows + row];
-            const uint32_t dst = dst0 + (uint32_t)smx_chunk_off(row, chunk, kSmxRows);
-            if (r != 0xFFFFFFFFu) cp_async<16>(dst, Xg + (size_t)r * p + f_first + chunk * 8);
-            else st_shared_zero16(dst);  // an empty slot must contribute nothing
+        if (warp >= kSmxRows / 32) {
+            // Producer warps take 256/16 = 16 row slots each: one warp can keep only a few copy instructions in
+            // flight, so many warps share the gather.  Lanes 0..15 evaluate the shuffle for one slot each; then the
+            // warp copies the 16 rows one after the other, lanes taking consecutive 16-byte chunks.
+            constexpr int kProducers = kSmxThreads / 32 - kSmxRows / 32;
+            constexpr int kSlots = kSmxRows / kProducers;
+            const int lane = tid & 31;
+            const bool active = lane < NP * 8;
+            const uint32_t dst_lane = smem_u32(xbuf[b]) + (uint32_t)((lane >> 3) * kSmxRows * 128);
+            const __nv_bfloat16* src_lane = Xg + f_first + lane * 8;
+            {
+                const int slot0 = (warp - kSmxRows / 32) * kSlots;
+                const int slot = slot0 + lane;
+                uint32_t r = 0xFFFFFFFFu;
+                int label = -1;
+                if (lane < kSlots && (uint32_t)slot < nm) {
+                    r = perm_index(lo + (uint32_t)slot, dom, rk);
+                    if (slot / RO == rank) label = P.y[r];
+                }
+#pragma unroll 4
+                for (int i = 0; i < kSlots; ++i) {
+                    const uint32_t ri = __shfl_sync(0xFFFFFFFFu, r, i);
+                    const int row = slot0 + i;
+                    const uint32_t dst = dst_lane + (uint32_t)(row * 128 + (((lane & 7) ^ (row & 7)) << 4));
+                    if (active) {
+                        if (ri != 0xFFFFFFFFu) cp_async<16>(dst, src_lane + (size_t)ri * p);
+                        else st_shared_zero16(dst);  // an empty slot must contribute nothing
+                    }
+                }
+                // labels of the slots this CTA owns, for the step that will read buffer b
+                if (lane < kSlots && slot / RO == rank) lab[b * kSmxRows + slot % RO] = label;
+            }
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
-
     if (total_steps > 0) {
         gather(0, 0);
-        if (tid < RO) lab[tid] = next_label;
     }
     uint32_t mma_phase = 0;
 
@@ -301,15 +319,26 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
         const int b = (int)(step & 1u);
         uint32_t lo, nm;
         step_rows(step, lo, nm);
-        // start fetching the next step's rows into the other buffer (its last reader finished a step ago)
-        if (step + 1 < total_steps) {
-            gather(step + 1, b ^ 1);
-            asm volatile("cp.async.wait_group 1;" ::: "memory");
-        } else {
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-        }
+#ifdef BMGD_TRACE
+        const uint32_t step_count = step;
+#endif
+        BMGD_STAMP(0);
+        asm volatile("cp.async.wait_group 0;" ::: "memory");  // this step's rows (issued during the previous step)
         if constexpr (USE_TC) fence_async_proxy();  // cp.async and st.shared wrote what the tensor core will read
         __syncthreads();
+        BMGD_STAMP(1);
+
+        if (warp >= kSmxRows / 32) {
+            // ---- producer warps: arrive at the first barrier at once, fetch the next step's rows into the other
+            //      buffer (its last reader, the previous step's backward contraction, has finished), then join
+            //      the second barrier
+            if (S > 1) cluster_arrive_release(); else named_arrive(1, kSmxThreads);
+            if (step + 1 < total_steps) gather(step + 1, b ^ 1);
+            __syncwarp();
+            if (S > 1) { cluster_wait_acquire(); cluster_arrive_release(); cluster_wait_acquire(); }
+            else named_sync(2, kSmxThreads);
+            continue;
+        }
 
         // ---- forward: partial logits of row slot `tid` (threads 0..255) over this CTA's predictors
         float z[kSmxClasses];
@@ -355,6 +384,7 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
             }
         }
 
+        BMGD_STAMP(2);
         // ---- reduce-scatter of the partial logits: row slot -> the CTA that owns it
         if (tid < kSmxRows) {
             const int owner = tid / RO, rloc = tid % RO;
@@ -363,8 +393,9 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
 #pragma unroll
             for (int c4 = 0; c4 < 4; ++c4) st_cluster_v4(dst + c4 * 16, z[c4 * 4], z[c4 * 4 + 1], z[c4 * 4 + 2], z[c4 * 4 + 3]);
         }
-        if (S > 1) { __syncwarp(); cluster_arrive_release(); cluster_wait_acquire(); } else __syncthreads();
+        if (S > 1) { __syncwarp(); cluster_arrive_release(); cluster_wait_acquire(); } else named_sync(1, kSmxThreads);
 
+        BMGD_STAMP(3);
         // ---- softmax and residual for the rows this CTA owns; push R to every peer
         for (int r0 = 0; r0 < RO; r0 += 16) {
             if (tid < 256) {
@@ -382,23 +413,30 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
                 for (int off = 8; off > 0; off >>= 1) den += __shfl_xor_sync(0xFFFFFFFFu, den, off);
                 float res = 0.f;
                 if (live && (uint32_t)slot < nm) res = __fdividef(e, den) - (c == lab[b * kSmxRows + rloc] ? 1.f : 0.f);
-                const unsigned short rb16 = __bfloat16_as_ushort(__float2bfloat16_rn(res));
                 // tensor-core path: R^T as B operand, [row panel of 64][class][128 B] swizzled; otherwise [row][class]
                 const int off = USE_TC ? (smx_chunk_off(c, slot >> 3, kSmxClasses) + (slot & 7) * 2) : (slot * kSmxClasses + c) * 2;
-                const uint32_t dst_local = smem_u32(rbuf + off);
-                if (S > 1) {
-                    for (int peer = 0; peer < S; ++peer) st_cluster_u16(map_to_cta(dst_local, (uint32_t)peer), rb16);
-                } else {
-                    *reinterpret_cast<unsigned short*>(rbuf + off) = rb16;
-                }
+                *reinterpret_cast<__nv_bfloat16*>(rbuf + off) = __float2bfloat16_rn(res);
             }
         }
-        // labels of the next step's rows were fetched while this step ran
-        if (tid < RO) lab[(b ^ 1) * kSmxRows + tid] = next_label;
+        if (S > 1) {
+            // the owned part of R is 2*RO chunks of 16 bytes: copy each to every peer
+            named_sync(3, kSmxRows);
+            if (tid < 2 * RO) {
+                const int per_class = RO / 8;
+                const int off = USE_TC ? smx_chunk_off(tid / per_class, rank * per_class + tid % per_class, kSmxClasses)
+                                       : (rank * RO * kSmxClasses * 2 + tid * 16);
+                const float4 v = *reinterpret_cast<const float4*>(rbuf + off);
+                const uint32_t dst_local = smem_u32(rbuf + off);
+                for (int peer = 0; peer < S; ++peer)
+                    if (peer != rank) st_cluster_v4(map_to_cta(dst_local, (uint32_t)peer), v.x, v.y, v.z, v.w);
+            }
+        }
+        BMGD_STAMP(4);
         if constexpr (USE_TC) fence_async_proxy();
-        if (S > 1) { __syncwarp(); cluster_arrive_release(); cluster_wait_acquire(); } else __syncthreads();
+        if (S > 1) { __syncwarp(); cluster_arrive_release(); cluster_wait_acquire(); } else named_sync(2, kSmxThreads);
         if constexpr (USE_TC) fence_async_proxy();  // the peers' residuals arrived through the generic proxy
 
+        BMGD_STAMP(5);
         // ---- backward: gradient rows of this CTA's predictors
         float gr[kSmxClasses];
 #pragma unroll
@@ -436,6 +474,7 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
             }
         }
 
+        BMGD_STAMP(6);
         // ---- update of W_slice and of its bf16 copy
         const float scale = (float)((nm == n) ? P.scale_full : P.scale_last);
         if (owns_w) {
@@ -443,6 +482,7 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
             for (int c = 0; c < kSmxClasses; ++c) w[c] = fmaf(-scale, gr[c], w[c]);
         }
         write_wt();
+        BMGD_STAMP(7);
         // the next iteration's barrier orders these writes, and the end of the reads of xbuf[b], before their next use
     }
 
