@@ -205,6 +205,12 @@ int bmgd_get_stats(bmgd_t* h, bmgd_stats* out);
 int bmgd_debug_perm(bmgd_t* h, uint64_t seed, uint32_t chain, uint32_t round, uint32_t N0,
                     uint32_t* out_host);
 
+/* Launch, on the compute stream, a one-thread kernel that waits with the step kernels' bounded-wait protocol for
+ * something that never happens, with a budget of budget_ms (at most 1000).  The wait gives up, the kernel returns,
+ * and the next synchronising call reports BMGD_ERR_TIMEOUT once; the handle stays usable.  For testing the error
+ * path without hanging or faulting a GPU.  Not for softmax handles. */
+int bmgd_debug_wait_timeout(bmgd_t* h, double budget_ms);
+
 /* Text for a bmgd_status; never NULL. */
 const char* bmgd_strerror(int status);
 /* cudaError_t of the last failed runtime call on this handle (0 if none). */

@@ -31,7 +31,7 @@ EXPORTS = (
     "bmgd_config_init", "bmgd_workspace_bytes", "bmgd_create", "bmgd_create_ex", "bmgd_destroy",
     "bmgd_load_buffer", "bmgd_run_rounds", "bmgd_run_rounds_resident", "bmgd_sync", "bmgd_get_theta",
     "bmgd_set_theta", "bmgd_get_stats", "bmgd_debug_perm", "bmgd_strerror", "bmgd_last_cuda_error",
-    "bmgd_version", "bmgd_run_rounds_noalloc",
+    "bmgd_version", "bmgd_run_rounds_noalloc", "bmgd_debug_wait_timeout",
 )
 
 
@@ -103,6 +103,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.bmgd_strerror.argtypes = [ctypes.c_int]; L.bmgd_strerror.restype = ctypes.c_char_p
     L.bmgd_last_cuda_error.argtypes = [vp]
     L.bmgd_version.argtypes = []
+    L.bmgd_debug_wait_timeout.argtypes = [vp, dbl]
     L.bmgd_run_rounds_noalloc.argtypes = [vp, vp, i64, i32, i32, i32, i32, vp, i32, i32, dbl, u64, vp]
     for name in EXPORTS:
         if getattr(L, name).restype is None or name in ("bmgd_strerror",):
@@ -247,6 +248,9 @@ class Bmgd:
         self._check(self._lib.bmgd_debug_perm(self._h, int(seed) & 0xFFFFFFFFFFFFFFFF, chain, rnd, N0,
                                               out.ctypes.data), "bmgd_debug_perm")
         return out
+
+    def debug_wait_timeout(self, budget_ms: float) -> None:
+        self._check(self._lib.bmgd_debug_wait_timeout(self._h, float(budget_ms)), "bmgd_debug_wait_timeout")
 
     def close(self) -> None:
         if getattr(self, "_h", None) is not None and self._h:

@@ -220,31 +220,45 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     const bool pre = var->kch * var->vec <= 16;
     const int pitch = pcap * eb + 16;
 
-    // cluster size
+    // Cluster size.  Measured on B200: a step costs one cluster barrier (about 0.6-0.9 us) inside one cluster, and
+    // about 2.5 us more once partial sums have to cross clusters through L2, while a sub-pass of spp rows costs about
+    // 0.35 us.  So a chain gets the largest cluster the device admits and stays inside it unless a CTA would have to
+    // sweep many sub-passes per step.
     int S = c.cluster_size;
     if (S == 0) {
         if (c.Rc > 1) S = std::min(8, floor_pow2(std::max(1, h->sm_count / c.Rc)));
-        else S = 8;
+        else S = 16;
         // do not spread a mini-batch thinner than 8 rows per CTA
         while (S > 1 && n / S < 8) S /= 2;
     }
-    L.S = S;
 
     // How many clusters can be resident depends on shared memory, which depends on the ring; ask with
     // the largest ring we would use (a smaller one can only admit more).
-    const int fixed_smem = bmgdk::glm_smem_plan(warps, gpw, pre, 1, 0, pcap, eb, S).total_bytes;
-    const int ring_budget = std::min(h->smem_optin - fixed_smem, 160 * 1024);
-    if (ring_budget < spp * pitch) return BMGD_ERR_UNIMPLEMENTED;
-    const int probe_smem = fixed_smem + ring_budget;
-    BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn, cudaFuncAttributeMaxDynamicSharedMemorySize, probe_smem));
-    if (S > 8) BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
-    int max_clusters = h->sm_count;
-    if (S > 1) {
-        int rc = max_active_clusters(h, var->fn, S, L.threads, probe_smem, &max_clusters);
-        if (rc != BMGD_OK) return rc;
+    int max_clusters = 0, fixed_smem = 0, ring_budget = 0;
+    for (;;) {
+        fixed_smem = bmgdk::glm_smem_plan(warps, gpw, pre, 1, 0, pcap, eb, S).total_bytes;
+        ring_budget = std::min(h->smem_optin - fixed_smem, 160 * 1024);
+        if (ring_budget < 2 * spp * pitch) {  // the per-peer exchange buffers of a large cluster leave no room for rows
+            if (c.cluster_size == 0 && S > 1) { S /= 2; continue; }
+            return BMGD_ERR_UNIMPLEMENTED;
+        }
+        const int probe_smem = fixed_smem + ring_budget;
+        BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn, cudaFuncAttributeMaxDynamicSharedMemorySize, probe_smem));
+        BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn, cudaFuncAttributeNonPortableClusterSizeAllowed, S > 8 ? 1 : 0));
+        max_clusters = h->sm_count;
+        if (S > 1) {
+            int rc = max_active_clusters(h, var->fn, S, L.threads, probe_smem, &max_clusters);
+            if (rc != BMGD_OK) {
+                if (c.cluster_size == 0 && S > 8) { S = 8; continue; }  // clusters of 16 are optional in hardware
+                return rc;
+            }
+        }
+        if (max_clusters < 1 && c.cluster_size == 0 && S > 8) { S = 8; continue; }
+        break;
     }
     if (max_clusters < 1) return BMGD_ERR_LAUNCH;
     max_clusters = std::min(max_clusters, kMaxClustersForExchange);
+    L.S = S;
 
     if (c.Rc > 1 && c.ctas_per_chain == 0) {
         L.cpc = 1;
@@ -255,9 +269,10 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
             if (c.ctas_per_chain % S != 0) return BMGD_ERR_ARG;
             cpc = c.ctas_per_chain / S;
         } else {
-            cpc = std::max(1, std::min(max_clusters, n / (8 * S)));
+            const int sp1 = (n + S * spp - 1) / (S * spp);  // sub-passes per step with a single cluster
+            cpc = sp1 <= 6 ? 1 : std::min(max_clusters, (sp1 + 1) / 2);
         }
-        cpc = std::min(cpc, bmgdk::kMaxCpc);
+        cpc = std::max(1, std::min(cpc, bmgdk::kMaxCpc));
         if (cpc > max_clusters) return BMGD_ERR_LAUNCH;
         L.cpc = cpc;
         L.nteams = std::max(1, std::min(c.Rc, max_clusters / cpc));
@@ -819,6 +834,20 @@ int bmgd_run_rounds_noalloc(const void* dev_x, const void* dev_y, int64_t rows, 
     }
     if (status[0] != 0) return status[0];
     if (status[1] != 0) return BMGD_ERR_TIMEOUT;
+    return BMGD_OK;
+}
+
+int bmgd_debug_wait_timeout(bmgd_t* h, double budget_ms) {
+    if (!h || !(budget_ms > 0) || budget_ms > 1000.0) return BMGD_ERR_ARG;
+    if (h->cfg.loss == BMGD_LOSS_SOFTMAX) return BMGD_ERR_UNIMPLEMENTED;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return cuda_fail(h, cudaErrorInvalidDevice);
+    // tag 0xFFFFFFFF is never written: the host keeps step tags below 0xFFFFFFF0
+    bmgdk::wait_probe_kernel<<<1, 1, 0, h->compute>>>(reinterpret_cast<const unsigned long long*>(h->base + h->lay.ll),
+                                                    0xFFFFFFFFu, (unsigned long long)(budget_ms * 1e6),
+                                                    reinterpret_cast<int*>(h->base + h->lay.status));
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(h, e);
     return BMGD_OK;
 }
 

@@ -137,7 +137,7 @@ __device__ __forceinline__ void st_packet(unsigned long long* p, unsigned long l
 }
 __device__ __forceinline__ unsigned long long ld_packet(const unsigned long long* p) {
     unsigned long long v;
-    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p));
     return v;
 }
 __device__ __forceinline__ unsigned long long global_ns() {
@@ -193,12 +193,15 @@ __host__ __device__ inline GlmSmemPlan glm_smem_plan(int warps, int gpw, bool pr
 }
 
 #ifdef BMGD_TRACE
-// Debug build only: clock stamps of CTA 0 at the phase boundaries of its first steps.
+// Debug build only: clock stamps of one CTA at the phase boundaries of its first steps.
+#ifndef BMGD_TRACE_BLOCK
+#define BMGD_TRACE_BLOCK 0
+#endif
 constexpr int kTraceSteps = 64, kTracePhases = 16;
 __device__ long long g_trace[kTraceSteps * kTracePhases];
 #define BMGD_STAMP(ph)                                                                              \
     do {                                                                                            \
-        if (blockIdx.x == 0 && threadIdx.x == 0 && step_count < (uint32_t)kTraceSteps)              \
+        if (blockIdx.x == BMGD_TRACE_BLOCK && threadIdx.x == 0 && step_count < (uint32_t)kTraceSteps) \
             g_trace[step_count * kTracePhases + (ph)] = clock64();                                  \
     } while (0)
 #else
@@ -535,7 +538,6 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                         }
                         __syncwarp();
                         cluster_arrive_release();
-                        issue_one();
                         cluster_wait_acquire();
                     }
                     BMGD_STAMP(4);
@@ -554,7 +556,7 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                                           ((unsigned long long)tag << 32) | Words<T>::get(mine_sum, w));
                         }
                     }
-                    if (S == 1) issue_one();
+                    BMGD_STAMP(12);
 #pragma unroll
                     for (int i = 0; i < FPT; ++i) {
                         const int j = tid + i * nthreads;
@@ -564,15 +566,21 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                         unsigned long long t0 = 0;
                         uint32_t spins = 0;
                         while (!aborted) {
+                            // all loads first, all tag checks after: a check between two loads would make the
+                            // second load wait for the first one's round trip to L2
+#pragma unroll
+                            for (int k = 0; k < kMaxCpc; ++k) {
+                                if (k < cpc) {
+#pragma unroll
+                                    for (int w = 0; w < NW; ++w) v[k][w] = ld_packet(slot + (size_t)k * P.ll_stride + f * NW + w);
+                                }
+                            }
                             bool ok = true;
 #pragma unroll
                             for (int k = 0; k < kMaxCpc; ++k) {
                                 if (k < cpc) {
 #pragma unroll
-                                    for (int w = 0; w < NW; ++w) {
-                                        v[k][w] = ld_packet(slot + (size_t)k * P.ll_stride + f * NW + w);
-                                        ok &= ((uint32_t)(v[k][w] >> 32) == tag);
-                                    }
+                                    for (int w = 0; w < NW; ++w) ok &= ((uint32_t)(v[k][w] >> 32) == tag);
                                 }
                             }
                             if (ok) break;
@@ -586,6 +594,12 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                                 }
                             }
                         }
+#ifdef BMGD_TRACE
+                        if (blockIdx.x == BMGD_TRACE_BLOCK && tid == 0 && step_count < (uint32_t)kTraceSteps) {
+                            g_trace[step_count * kTracePhases + 13] = clock64();
+                            g_trace[step_count * kTracePhases + 14] = spins;
+                        }
+#endif
                         T s = T(0);
                         if (!aborted) {
 #pragma unroll
@@ -606,11 +620,15 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                         }
                     }
                     BMGD_STAMP(5);
+                    // The copies for a later stage go out only now: issued earlier they would sit in front of the
+                    // packet stores and polls on the same load/store path and delay the exchange by their drain time.
+                    __syncwarp();
                     if (S > 1) {
-                        __syncwarp();
                         cluster_arrive_release();
+                        issue_one();
                         cluster_wait_acquire();
                     } else {
+                        issue_one();
                         __syncthreads();
                     }
                 }
@@ -651,6 +669,26 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
         }
     }
     cp_async_wait_all();
+}
+
+// Waits, with the step kernel's protocol, for a packet tag that nobody writes: the wait must run out of its
+// budget, record BMGD_ERR_TIMEOUT in the status word, raise the abort flag and return.  For testing the error path.
+__global__ void wait_probe_kernel(const unsigned long long* packet, uint32_t tag, unsigned long long timeout_ns, int* status) {
+    unsigned long long t0 = 0;
+    uint32_t spins = 0;
+    bool aborted = false;
+    while (!aborted) {
+        if ((uint32_t)(ld_packet(packet) >> 32) == tag) break;
+        if ((++spins & 0x3FFu) == 0u) {
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > timeout_ns || ((volatile int*)status)[1] != 0) {
+                atomicCAS(status, 0, kStatusTimeout);
+                atomicExch(status + 1, 1);
+                aborted = true;
+            }
+        }
+    }
 }
 
 // Writes out[j] = pi(j) for one (seed, chain, round): the shuffle exactly as the step kernel uses it.

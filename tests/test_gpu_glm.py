@@ -186,3 +186,25 @@ def test_cfg3_one_full_buffer_default_shape():
     """One full cfg3 buffer (1,000,000 x 200 logistic, n=4,096, 245 steps per round), two rounds."""
     w = WORKLOADS["cfg3"].scaled(N=1_000_000, K=1, T=2, epochs=1)
     check(w, buffers_of(w), mode="resident")
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_handle_stays_usable():
+    """Failure detection without a GPU fault: a bounded wait gives up after its budget, the status word carries
+    BMGD_ERR_TIMEOUT to the next synchronising call, and the same handle then computes correctly."""
+    import time
+    from paper_2312_08728_b200.binding import Bmgd, BmgdError, ERR_TIMEOUT, FLAG_NO_SLOTS
+    w = SMALL
+    bufs = buffers_of(w)
+    X, y = [t.cuda() for t in bufs[0]]
+    with Bmgd(w.N, w.p, w.K, loss=w.loss, dtype=w.dtype, flags=FLAG_NO_SLOTS) as h:
+        t0 = time.perf_counter()
+        h.debug_wait_timeout(50.0)
+        with pytest.raises(BmgdError) as e:
+            h.sync()
+        assert e.value.status == ERR_TIMEOUT
+        assert 0.04 <= time.perf_counter() - t0 < 5.0
+        h.sync()  # reported once, then cleared
+        h.run_rounds_resident(X, y, w.T, w.n, w.lr, inputs.buffer_seed(w.seed, 0, 0, w.K))
+        theta = h.get_theta()
+    want = oracle_job(w.scaled(K=1, N=w.N0), bufs[:1])[0]
+    assert rel_l2(theta[0], want) <= 1e-4
