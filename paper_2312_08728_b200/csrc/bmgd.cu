@@ -284,7 +284,8 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     // sub-passes per ring stage: two or more let a group keep two rows in flight and amortise the per-stage
     // bookkeeping; measured on B200, two stages of two sub-passes beat four stages of one when rows come from L2
     const int subpass_bytes = spp * pitch;
-    int rb = c.subpasses_per_stage ? c.subpasses_per_stage : 2;
+    // narrow rows (at most 32 bytes per lane) are swept four sub-passes at a time by the kernel, others two
+    int rb = c.subpasses_per_stage ? c.subpasses_per_stage : ((var->kch * 16 <= 32) ? 4 : 2);
     rb = std::min(rb, var->lpr);
     rb = floor_pow2(std::max(1, std::min(rb, subpasses)));
     while (rb > 1 && 2 * rb * subpass_bytes > ring_budget) rb /= 2;

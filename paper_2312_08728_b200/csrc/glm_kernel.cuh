@@ -448,6 +448,14 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                     if (++cs_slot == D) cs_slot = 0;
                     int nsub = min(sp_left, RB);
                     sp_left -= nsub;
+                    if constexpr (NV * (int)sizeof(T) <= 32) {  // narrow rows: four independent rows in flight per group
+                        for (; nsub >= 4; nsub -= 4, rowp += 4 * subpass_bytes) {
+                            row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, y_rel, th, gacc);
+                            row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + subpass_bytes, y_rel, th, gacc);
+                            row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + 2 * subpass_bytes, y_rel, th, gacc);
+                            row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + 3 * subpass_bytes, y_rel, th, gacc);
+                        }
+                    }
                     for (; nsub >= 2; nsub -= 2, rowp += 2 * subpass_bytes) {  // two independent rows in flight per group
                         row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, y_rel, th, gacc);
                         row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + subpass_bytes, y_rel, th, gacc);
