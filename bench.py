@@ -52,6 +52,7 @@ def parse_args():
     ap.add_argument("--threads", type=int, default=0)
     ap.add_argument("--depth", type=int, default=0)
     ap.add_argument("--subpasses", type=int, default=0, help="sub-passes per ring stage")
+    ap.add_argument("--bulk-rows", type=int, default=-1, help="1: fetch rows by cp.async.bulk, 0: by cp.async chunks, -1: library default")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
@@ -248,8 +249,9 @@ def config_of(args, w):
 
 def run_ours(args, w):
     import numpy as np
-    from paper_2312_08728_b200.binding import Bmgd, FLAG_NO_SLOTS, FLAG_TIMING
+    from paper_2312_08728_b200.binding import Bmgd, FLAG_NO_SLOTS, FLAG_TIMING, FLAG_BULK_ROWS
     rank, world, local = dist_env()
+    extra_flags = FLAG_BULK_ROWS if args.bulk_rows == 1 else 0
     multi = world > 1
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
@@ -274,7 +276,7 @@ def run_ours(args, w):
     resident = [(x.to(dev), y.to(dev)) for x, y in host]
     with torch.cuda.stream(stream):
         h = Bmgd(w.N, w.p, w.K, loss=w.loss, dtype=w.dtype, C=w.C, Rc=w.Rc, device=local,
-                 flags=FLAG_NO_SLOTS | FLAG_TIMING, use_torch_stream=True, **shape)
+                 flags=FLAG_NO_SLOTS | FLAG_TIMING | extra_flags, use_torch_stream=True, **shape)
 
         def step(i):
             x, y = resident[i % nb]
@@ -316,7 +318,7 @@ def run_ours(args, w):
         copy = torch.cuda.Stream(dev)
         with torch.cuda.stream(stream):
             h = Bmgd(w.N, w.p, w.K, loss=w.loss, dtype=w.dtype, C=w.C, Rc=w.Rc, device=local,
-                     flags=FLAG_TIMING, use_torch_stream=True, **shape)
+                     flags=FLAG_TIMING | extra_flags, use_torch_stream=True, **shape)
             total = args.warmup + args.steps
             e2e_s0 = None
             slot = h.load_buffer(*pinned[0], stream=copy)

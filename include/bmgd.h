@@ -61,6 +61,8 @@ enum {
                                        assumption under which Eq. (3.1)-(3.3) are derived */
     BMGD_FLAG_NO_SLOTS = 2u,        /* allocate no buffer slots: only bmgd_run_rounds_resident is used */
     BMGD_FLAG_TIMING = 4u,          /* record CUDA events round every launch and copy (bmgd_get_stats) */
+    BMGD_FLAG_BULK_ROWS = 16u,      /* linear/logistic: fetch each row with one bulk copy (cp.async.bulk) instead of
+                                       16-byte cp.async chunks; needs rows that are 16-byte multiples */
     BMGD_FLAG_SOFTMAX_CUDA_CORES = 8u /* softmax: run the two contractions on the CUDA cores, not the tensor cores
                                        (same bf16 inputs; for cross-checking the tensor-core path) */
 };

@@ -25,6 +25,7 @@ FLAG_FIXED_PARTITION = 1
 FLAG_NO_SLOTS = 2
 FLAG_TIMING = 4
 FLAG_SOFTMAX_CUDA_CORES = 8
+FLAG_BULK_ROWS = 16
 
 # every symbol include/bmgd.h declares
 EXPORTS = (

@@ -372,6 +372,7 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
     P.ll_stride = c.p * 2;
     P.tag_base = (uint32_t)h->tag_base;
     P.fixed_partition = (c.flags & BMGD_FLAG_FIXED_PARTITION) ? 1 : 0;
+    P.bulk_rows = (aligned16 && (c.flags & BMGD_FLAG_BULK_ROWS)) ? 1 : 0;
     if ((int64_t)L.nteams * L.cpc > kMaxClustersForExchange) return BMGD_ERR_LAUNCH;
 
     cudaLaunchConfig_t lc{};

@@ -63,6 +63,7 @@ struct GlmParams {
     int ll_stride;        // packets per cluster slot
     uint32_t tag_base;
     int fixed_partition;
+    int bulk_rows;        // rows travel as one bulk copy each (cp.async.bulk) instead of 16-byte cp.async chunks
 };
 
 // ---------------------------------------------------------------- small PTX wrappers
@@ -132,6 +133,32 @@ __device__ __forceinline__ void cluster_arrive_release() {
 __device__ __forceinline__ void cluster_wait_acquire() {
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// ---- mbarriers (8 bytes of shared memory each) and bulk copies
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// the arrival happens once every cp.async this thread has issued so far has landed
+__device__ __forceinline__ void mbar_arrive_after_copies(uint32_t bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+// generic-proxy writes to shared memory become ordered with the bulk copies' writes and the tensor core's reads
+__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// one row, global -> shared, completion counted in bytes on `bar`; addresses and size are 16-byte multiples
+__device__ __forceinline__ void bulk_copy_row(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
 __device__ __forceinline__ void st_packet(unsigned long long* p, unsigned long long v) {
     asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
@@ -172,7 +199,7 @@ template <> struct Words<double> {
 struct GlmSmemPlan {
     int pitch;             // bytes from one ring row to the next: the full predictor capacity, then 16 bytes for y
     int warp_stage_bytes;  // one warp's share of one ring stage
-    int ring_bytes;
+    int ring_off, ring_bytes;
     int gpart_rows;        // partial-gradient rows summed per CTA
     int gpart_off, cpart_off, gfin_off;
     int total_bytes;
@@ -183,9 +210,10 @@ __host__ __device__ inline GlmSmemPlan glm_smem_plan(int warps, int gpw, bool pr
     GlmSmemPlan s;
     s.pitch = pcap * elem_bytes + 16;
     s.warp_stage_bytes = rb * gpw * s.pitch;
+    s.ring_off = 1024;  // room for one mbarrier per (warp, stage) in front of the ring
     s.ring_bytes = warps * depth * s.warp_stage_bytes;
     s.gpart_rows = prereduce ? warps : warps * gpw;
-    s.gpart_off = s.ring_bytes;
+    s.gpart_off = s.ring_off + s.ring_bytes;
     s.cpart_off = s.gpart_off + s.gpart_rows * pcap * elem_bytes;
     s.gfin_off = s.cpart_off + 2 * S * pcap * elem_bytes;
     s.total_bytes = s.gfin_off + pcap * elem_bytes;
@@ -333,7 +361,9 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
 
     const GlmSmemPlan plan = glm_smem_plan(W, GPW, PRE, RB, D, PCAP, (int)sizeof(T), S);
     const int pitch = plan.pitch;
-    unsigned char* my_ring = smem + warp * D * plan.warp_stage_bytes;
+    unsigned char* my_ring = smem + plan.ring_off + warp * D * plan.warp_stage_bytes;
+    const uint32_t my_bars = smem_u32(smem) + (uint32_t)(warp * D * 8);  // one mbarrier per stage of this warp's ring
+    const bool bulk = P.bulk_rows != 0;
     T* gpart = reinterpret_cast<T*>(smem + plan.gpart_off);
     T* cpart = reinterpret_cast<T*>(smem + plan.cpart_off);
     T* gfin = reinterpret_cast<T*>(smem + plan.gfin_off);
@@ -355,7 +385,10 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
     uint32_t to_issue = (uint32_t)nch * (uint32_t)T_rounds * M * (uint32_t)passes;  // the host keeps this below 2^32
 
     // zero all of shared memory once: row tails beyond p and never-written slots must read as zero
-    for (int i = tid * 16; i < plan.total_bytes; i += nthreads * 16) st_shared_zero16(smem_u32(smem + i));
+    for (int i = plan.ring_off + tid * 16; i < plan.total_bytes; i += nthreads * 16) st_shared_zero16(smem_u32(smem + i));
+    if (tid < W * D) mbar_init(smem_u32(smem) + (uint32_t)(tid * 8), 33u);  // 32 lanes after their copies + the byte count
+    fence_barrier_init();
+    fence_async_proxy();  // bulk copies will overwrite bytes zeroed here
     __syncthreads();
     if (S > 1) {  // peers must be running (and zeroed) before anyone writes into their shared memory
         cluster_arrive_release();
@@ -373,6 +406,8 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
         if (to_issue != 0u) {
             --to_issue;
             uint32_t dst = smem_u32(my_ring + pf_slot * plan.warp_stage_bytes) + lane_off;
+            const uint32_t pf_bar = my_bars + (uint32_t)(pf_slot * 8);
+            int pf_rows_in_stage = 0;
             int sp = pf_sidx * RB;
             for (int r = 0; r < RB; ++r, ++sp, dst += subpass_bytes) {
                 const int bi = sp & (LPR - 1);
@@ -383,8 +418,15 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                 if ((uint32_t)sp < pfs.nsp) {  // otherwise the whole warp skips this sub-pass, here and in the compute loop
                     const uint32_t row = __shfl_sync(0xFFFFFFFFu, pf_rows, bi * GPW + grp);
                     if (row != kNoRow) {
-                        cp_async_chunks<CB, LPR * CB, 0, KCH>(dst, Xb + (size_t)row * row_bytes, kmask);
-                        cp_async_at<(int)sizeof(T), 0>(dst + y_rel, yb + row, sub == 0 ? 1u : 0u);
+                        if (bulk) {
+                            if (sub == 0) {  // one bulk copy per row; its bytes are counted on the stage's mbarrier
+                                bulk_copy_row(dst, Xb + (size_t)row * row_bytes, row_bytes, pf_bar);
+                                cp_async<(int)sizeof(T)>(dst + YOFF, yb + row);
+                            }
+                        } else {
+                            cp_async_chunks<CB, LPR * CB, 0, KCH>(dst, Xb + (size_t)row * row_bytes, kmask);
+                            cp_async_at<(int)sizeof(T), 0>(dst + y_rel, yb + row, sub == 0 ? 1u : 0u);
+                        }
                     } else {  // no row for this slot: it must contribute nothing
 #pragma unroll
                         for (int k = 0; k < KCH; ++k) {
@@ -393,7 +435,9 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                             else asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst + k * LPR * CB), "r"(0) : "memory");
                         }
                         if (sub == 0) st_shared_zero16(dst + y_rel);
+                        if (bulk) fence_async_proxy();  // a later bulk copy will overwrite these bytes
                     }
+                    if (bulk) pf_rows_in_stage += __popc(__ballot_sync(0xFFFFFFFFu, row != kNoRow && sub == 0));
                 }
             }
             if (++pf_sidx == passes) {
@@ -407,15 +451,20 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                 }
                 pfs = row_share(pf_m, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full, warp_first, spp_log2);
             }
+            if (bulk) {
+                if (lane == 0) mbar_arrive_expect_tx(pf_bar, (uint32_t)pf_rows_in_stage * row_bytes);
+                mbar_arrive_after_copies(pf_bar);
+            }
             if (++pf_slot == D) pf_slot = 0;
         }
-        cp_async_commit();
+        if (!bulk) cp_async_commit();
         __syncwarp();  // lanes walked the cycle for different lengths: meet again before any aligned barrier
     };
 
     for (int s = 0; s < D; ++s) issue_one();
 
     int cs_slot = 0;         // ring slot the compute cursor reads next
+    uint32_t cs_phase = 0;   // parity of that slot's mbarrier phase (bulk-copy mode)
     uint32_t step_count = 0; // steps this team has finished in this launch
     bool aborted = false;
 
@@ -442,10 +491,27 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
 
                 int sp_left = (int)sh.nsp;  // sub-passes of this step in which the warp still has rows
                 for (int sidx = 0; sidx < passes; ++sidx) {
-                    cp_async_wait_ring(D);
+                    if (bulk) {  // bounded wait on this warp's stage barrier
+                        const uint32_t bar = my_bars + (uint32_t)(cs_slot * 8);
+                        unsigned long long t0 = 0;
+                        uint32_t spins = 0;
+                        while (!aborted && !mbar_try_wait(bar, cs_phase)) {
+                            if ((++spins & 0x3Fu) == 0u) {
+                                const unsigned long long now = global_ns();
+                                if (t0 == 0) t0 = now;
+                                if (now - t0 > P.timeout_ns || ((volatile int*)P.status)[1] != 0) {
+                                    atomicCAS(P.status, 0, kStatusTimeout);
+                                    atomicExch(P.status + 1, 1);
+                                    aborted = true;
+                                }
+                            }
+                        }
+                    } else {
+                        cp_async_wait_ring(D);
+                    }
                     __syncwarp();
                     const unsigned char* rowp = my_ring + cs_slot * plan.warp_stage_bytes + lane_off;
-                    if (++cs_slot == D) cs_slot = 0;
+                    if (++cs_slot == D) { cs_slot = 0; cs_phase ^= 1u; }
                     int nsub = min(sp_left, RB);
                     sp_left -= nsub;
                     if constexpr (NV * (int)sizeof(T) <= 32) {  // narrow rows: four independent rows in flight per group

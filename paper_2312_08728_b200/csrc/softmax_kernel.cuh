@@ -97,18 +97,7 @@ __device__ __forceinline__ void named_sync(int id, int count) {
 }
 
 // ---------------------------------------------------------------- mbarrier and proxy helpers
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
-// generic-proxy writes to shared memory (st.shared, cp.async) become visible to the tensor core's reads
-__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// (mbar_init, mbar_try_wait, fence_barrier_init and fence_async_proxy come from glm_kernel.cuh)
 
 // Bounded wait: when the budget runs out the thread records BMGD_ERR_TIMEOUT, raises the abort flag and
 // stops waiting for the rest of the launch.

@@ -14,8 +14,8 @@ from helpers import TOL, buffers_of, gpu_job, oracle_job, rel_l2
 pytestmark = pytest.mark.gpu
 
 
-def check(w, buffers, chains=None, mode="slots", **shape):
-    theta, stats = gpu_job(w, buffers, mode=mode, **shape)
+def check(w, buffers, chains=None, mode="slots", flags=0, **shape):
+    theta, stats = gpu_job(w, buffers, mode=mode, flags=flags, **shape)
     want = oracle_job(w, buffers, chains=chains)
     worst = 0.0
     for c, th in want.items():
@@ -78,6 +78,31 @@ def test_launch_shapes_agree_with_the_oracle(shape):
     _, stats, _ = check(SMALL, buffers_of(SMALL), mode="resident", **shape)
     assert stats["cluster_size"] == shape["cluster_size"]
     assert stats["ctas_per_chain"] == shape["ctas_per_chain"]
+
+
+@pytest.mark.parametrize("shape", [
+    dict(cluster_size=1, ctas_per_chain=1),
+    dict(cluster_size=2, ctas_per_chain=12),
+    dict(cluster_size=8, ctas_per_chain=8, threads_per_cta=512),
+    dict(cluster_size=8, ctas_per_chain=16, pipeline_depth=2, subpasses_per_stage=4),
+    dict(cluster_size=16, ctas_per_chain=32),
+])
+def test_bulk_copy_rows_agree_with_the_oracle(shape):
+    """The same launches with every row fetched by one cp.async.bulk onto a per-warp mbarrier."""
+    from paper_2312_08728_b200.binding import FLAG_BULK_ROWS
+    check(SMALL, buffers_of(SMALL), mode="resident", flags=FLAG_BULK_ROWS, **shape)
+    w = WORKLOADS["cfg1"].scaled(N=4_000, K=2, epochs=1)
+    check(w, buffers_of(w), mode="slots", flags=FLAG_BULK_ROWS)
+
+
+def test_bulk_copy_rows_ragged_and_chains():
+    from paper_2312_08728_b200.binding import FLAG_BULK_ROWS
+    w = WORKLOADS["cfg3"].scaled(N=100_000, K=2, T=2, epochs=1)
+    check(w, buffers_of(w), flags=FLAG_BULK_ROWS)
+    w = WORKLOADS["cfg2"].scaled(N=60_000, K=3, T=2, epochs=1, Rc=8)
+    check(w, buffers_of(w), mode="resident", flags=FLAG_BULK_ROWS)
+    w = Workload("edge", LOSS_LINEAR, DTYPE_F64, N=257, p=6, K=1, n=3, T=2, lr=0.1, epochs=1, rho=0.5, seed=9)
+    check(w, buffers_of(w), mode="resident", flags=FLAG_BULK_ROWS)
 
 
 def test_cluster_of_sixteen_if_the_device_allows_it():
