@@ -207,6 +207,24 @@ int bmgd_get_stats(bmgd_t* h, bmgd_stats* out);
 int bmgd_debug_perm(bmgd_t* h, uint64_t seed, uint32_t chain, uint32_t round, uint32_t N0,
                     uint32_t* out_host);
 
+/*
+ * Partition of the whole sample into buffers (Algorithm 1, line 2: a fresh random partition {S_r,1..S_r,K} at the
+ * top of every pass r).  The partition of pass `pass` under `seed` is the same keyed bijection pi as the per-round
+ * shuffle, taken over [0, N) with the chain word 0xFFFFFFFF and the pass number as the round word; buffer k holds,
+ * in this order, rows pi(j) for k*N0 <= j < min((k+1)*N0, N), N0 = ceil(N/K).
+ *
+ * bmgd_partition_index writes pi(j) to *row.  bmgd_gather_buffer is the CPU side of the buffering step (Algorithm 1,
+ * line 3, "CPU starts preparing buffered data"): with `threads` host threads (<= 0: all hardware threads) it copies
+ * the rows of buffer k from host_x [N][row_bytes] and host_y [N][y_bytes] into stage_x, stage_y (at least N0 rows;
+ * pinned memory if they are handed to bmgd_load_buffer next) and writes the row count to *rows_out.  Pure host
+ * code: no GPU, no handle; safe to run from another thread while kernels and copies of earlier buffers are in flight.
+ * Errors: BMGD_ERR_ARG for null pointers or sizes out of range (N up to 2^31 - 1).
+ */
+int bmgd_partition_index(uint64_t seed, uint32_t pass, int64_t N, int64_t j, int64_t* row);
+int bmgd_gather_buffer(const void* host_x, const void* host_y, int64_t N, int64_t row_bytes, int64_t y_bytes,
+                       int32_t K, uint64_t seed, uint32_t pass, int32_t k, void* stage_x, void* stage_y,
+                       int32_t threads, int64_t* rows_out);
+
 /* Launch, on the compute stream, a one-thread kernel that waits with the step kernels' bounded-wait protocol for
  * something that never happens, with a budget of budget_ms (at most 1000).  The wait gives up, the kernel returns,
  * and the next synchronising call reports BMGD_ERR_TIMEOUT once; the handle stays usable.  For testing the error

@@ -32,7 +32,7 @@ EXPORTS = (
     "bmgd_config_init", "bmgd_workspace_bytes", "bmgd_create", "bmgd_create_ex", "bmgd_destroy",
     "bmgd_load_buffer", "bmgd_run_rounds", "bmgd_run_rounds_resident", "bmgd_sync", "bmgd_get_theta",
     "bmgd_set_theta", "bmgd_get_stats", "bmgd_debug_perm", "bmgd_strerror", "bmgd_last_cuda_error",
-    "bmgd_version", "bmgd_run_rounds_noalloc", "bmgd_debug_wait_timeout",
+    "bmgd_version", "bmgd_run_rounds_noalloc", "bmgd_debug_wait_timeout", "bmgd_partition_index", "bmgd_gather_buffer",
 )
 
 
@@ -105,6 +105,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.bmgd_last_cuda_error.argtypes = [vp]
     L.bmgd_version.argtypes = []
     L.bmgd_debug_wait_timeout.argtypes = [vp, dbl]
+    L.bmgd_partition_index.argtypes = [u64, u32, i64, i64, P(i64)]
+    L.bmgd_gather_buffer.argtypes = [vp, vp, i64, i64, i64, i32, u64, u32, i32, vp, vp, i32, P(i64)]
     L.bmgd_run_rounds_noalloc.argtypes = [vp, vp, i64, i32, i32, i32, i32, vp, i32, i32, dbl, u64, vp]
     for name in EXPORTS:
         if getattr(L, name).restype is None or name in ("bmgd_strerror",):
@@ -143,6 +145,38 @@ def run_rounds_noalloc(dev_x: torch.Tensor, dev_y: torch.Tensor, theta: torch.Te
                                    int(seed) & 0xFFFFFFFFFFFFFFFF, s)
     if rc != BMGD_OK:
         raise BmgdError(rc, "bmgd_run_rounds_noalloc")
+
+
+PARTITION_CHAIN = 0xFFFFFFFF  # chain word of the sample-level partition
+
+
+def partition_index(seed: int, epoch: int, N: int, j: int) -> int:
+    """Row of the sample that sits at position j of pass `epoch`'s random partition into buffers."""
+    out = ctypes.c_int64(-1)
+    rc = load_library().bmgd_partition_index(int(seed) & 0xFFFFFFFFFFFFFFFF, epoch, N, j, ctypes.byref(out))
+    if rc != BMGD_OK:
+        raise BmgdError(rc, "bmgd_partition_index")
+    return out.value
+
+
+def gather_buffer(host_x: torch.Tensor, host_y: torch.Tensor, K: int, seed: int, epoch: int, k: int,
+                  stage_x: torch.Tensor, stage_y: torch.Tensor, threads: int = 0) -> int:
+    """Gather buffer k of pass `epoch` from the whole host-resident sample into the staging tensors (host threads
+    inside the library; the GIL is released for the duration of the call).  Returns the number of rows."""
+    for t in (host_x, host_y, stage_x, stage_y):
+        if t.device.type != "cpu" or not t.is_contiguous():
+            raise ValueError("gather_buffer takes contiguous host tensors")
+    N = host_x.shape[0]
+    row_bytes = host_x.shape[1] * host_x.element_size()
+    if stage_x.shape[1] * stage_x.element_size() != row_bytes or stage_x.shape[0] < -(-N // K) or stage_y.shape[0] < -(-N // K):
+        raise ValueError("staging tensors are too small for a buffer")
+    rows = ctypes.c_int64(0)
+    rc = load_library().bmgd_gather_buffer(host_x.data_ptr(), host_y.data_ptr(), N, row_bytes, host_y.element_size(), K,
+                                           int(seed) & 0xFFFFFFFFFFFFFFFF, epoch, k, stage_x.data_ptr(),
+                                           stage_y.data_ptr(), threads, ctypes.byref(rows))
+    if rc != BMGD_OK:
+        raise BmgdError(rc, "bmgd_gather_buffer")
+    return rows.value
 
 
 class Bmgd:

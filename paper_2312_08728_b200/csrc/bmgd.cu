@@ -12,6 +12,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <thread>
 #include <vector>
 
 #include "glm_kernel.cuh"
@@ -836,6 +837,55 @@ int bmgd_run_rounds_noalloc(const void* dev_x, const void* dev_y, int64_t rows, 
     }
     if (status[0] != 0) return status[0];
     if (status[1] != 0) return BMGD_ERR_TIMEOUT;
+    return BMGD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Partition of the whole sample into buffers (Algorithm 1, line 2) and the CPU side of the buffering step
+// (line 3): gather the rows of one buffer of one pass into a staging buffer, with host threads.
+
+int bmgd_partition_index(uint64_t seed, uint32_t pass, int64_t N, int64_t j, int64_t* row) {
+    if (!row || N <= 0 || N > 0x7FFFFFFFll || j < 0 || j >= N) return BMGD_ERR_ARG;
+    const bmgdk::FeistelDomain dom = bmgdk::make_domain((uint32_t)N);
+    const bmgdk::RoundKeys rk = bmgdk::round_keys(seed, 0xFFFFFFFFu, pass);
+    *row = (int64_t)bmgdk::perm_index((uint32_t)j, dom, rk);
+    return BMGD_OK;
+}
+
+int bmgd_gather_buffer(const void* host_x, const void* host_y, int64_t N, int64_t row_bytes, int64_t y_bytes,
+                       int32_t K, uint64_t seed, uint32_t pass, int32_t k, void* stage_x, void* stage_y,
+                       int32_t threads, int64_t* rows_out) {
+    if (!host_x || !host_y || !stage_x || !stage_y || !rows_out) return BMGD_ERR_ARG;
+    if (N <= 0 || N > 0x7FFFFFFFll || row_bytes <= 0 || y_bytes <= 0 || K <= 0 || K > N || k < 0 || k >= K) return BMGD_ERR_ARG;
+    const int64_t N0 = (N + K - 1) / K;
+    const int64_t first = (int64_t)k * N0;
+    const int64_t rows = std::max<int64_t>(0, std::min(N0, N - first));
+    *rows_out = rows;
+    if (rows == 0) return BMGD_OK;
+    const bmgdk::FeistelDomain dom = bmgdk::make_domain((uint32_t)N);
+    const bmgdk::RoundKeys rk = bmgdk::round_keys(seed, 0xFFFFFFFFu, pass);
+    const unsigned char* sx = static_cast<const unsigned char*>(host_x);
+    const unsigned char* sy = static_cast<const unsigned char*>(host_y);
+    unsigned char* dx = static_cast<unsigned char*>(stage_x);
+    unsigned char* dy = static_cast<unsigned char*>(stage_y);
+    auto work = [&](int64_t lo, int64_t hi) {
+        for (int64_t i = lo; i < hi; ++i) {
+            const size_t src = (size_t)bmgdk::perm_index((uint32_t)(first + i), dom, rk);
+            std::memcpy(dx + (size_t)i * row_bytes, sx + src * (size_t)row_bytes, (size_t)row_bytes);
+            std::memcpy(dy + (size_t)i * y_bytes, sy + src * (size_t)y_bytes, (size_t)y_bytes);
+        }
+    };
+    int nt = threads > 0 ? threads : (int)std::thread::hardware_concurrency();
+    nt = (int)std::max<int64_t>(1, std::min<int64_t>(nt, rows / 1024 + 1));
+    if (nt == 1) { work(0, rows); return BMGD_OK; }
+    std::vector<std::thread> pool;
+    try {
+        for (int t = 0; t < nt; ++t) pool.emplace_back(work, rows * t / nt, rows * (t + 1) / nt);
+    } catch (...) {
+        for (auto& th : pool) th.join();
+        return BMGD_ERR_ALLOC;
+    }
+    for (auto& th : pool) th.join();
     return BMGD_OK;
 }
 

@@ -233,3 +233,39 @@ def test_a_wait_that_runs_out_is_reported_and_the_handle_stays_usable():
         theta = h.get_theta()
     want = oracle_job(w.scaled(K=1, N=w.N0), bufs[:1])[0]
     assert rel_l2(theta[0], want) <= 1e-4
+
+
+def test_algorithm_1_with_a_fresh_partition_of_the_sample_every_pass():
+    """All of Algorithm 1: every pass re-partitions the sample into K buffers (host gather into pinned staging
+    buffers, two in flight), every round re-partitions the buffer, theta is carried throughout."""
+    import oracle
+    from paper_2312_08728_b200.binding import Bmgd, PARTITION_CHAIN, gather_buffer
+    from helpers import ORACLE_LOSS
+    w = Workload("alg1", LOSS_LOGISTIC, DTYPE_F32, N=30_011, p=48, K=4, n=512, T=2, lr=0.3, epochs=3, seed=21)
+    X, y = inputs.make_rows(w, 0, w.N)
+    part_seed = 4242
+    N0 = w.N0
+    stage = [(torch.empty(N0, w.p).pin_memory(), torch.empty(N0).pin_memory()) for _ in range(2)]
+    copy = torch.cuda.Stream()
+    with Bmgd(w.N, w.p, w.K, loss=w.loss, dtype=w.dtype) as h:
+        order = [(e, k) for e in range(w.epochs) for k in range(w.K)]
+        def stage_and_load(i):
+            e, k = order[i]
+            sx, sy = stage[i % 2]
+            rows = gather_buffer(X, y, w.K, part_seed, e, k, sx, sy)
+            return h.load_buffer(sx[:rows], sy[:rows], stream=copy)
+        slot = stage_and_load(0)
+        for i, (e, k) in enumerate(order):
+            h.run_rounds(slot, w.T, w.n, w.lr, inputs.buffer_seed(w.seed, e, k, w.K))
+            if i + 1 < len(order):
+                copy.synchronize()  # the staging buffer about to be refilled must have left the host
+                slot = stage_and_load(i + 1)
+        theta = h.get_theta()[0]
+    th = np.zeros(w.p)
+    for e in range(w.epochs):
+        part = oracle.perm(part_seed, PARTITION_CHAIN, e, w.N).astype(np.int64)
+        for k in range(w.K):
+            rows = torch.from_numpy(part[k * N0:(k + 1) * N0])
+            oracle.run_rounds(ORACLE_LOSS[w.loss], X[rows].contiguous(), y[rows].contiguous(), th, w.T, w.n, w.lr,
+                              inputs.buffer_seed(w.seed, e, k, w.K))
+    assert rel_l2(theta, th) <= 1e-4
