@@ -52,7 +52,7 @@ def parse_args():
     ap.add_argument("--threads", type=int, default=0)
     ap.add_argument("--depth", type=int, default=0)
     ap.add_argument("--subpasses", type=int, default=0, help="sub-passes per ring stage")
-    ap.add_argument("--bulk-rows", type=int, default=-1, help="1: fetch rows by cp.async.bulk, 0: by cp.async chunks, -1: library default")
+    ap.add_argument("--producer-warps", type=int, default=0, help="warps per CTA that only fetch rows (0: library default)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
@@ -249,9 +249,9 @@ def config_of(args, w):
 
 def run_ours(args, w):
     import numpy as np
-    from paper_2312_08728_b200.binding import Bmgd, FLAG_NO_SLOTS, FLAG_TIMING, FLAG_BULK_ROWS
+    from paper_2312_08728_b200.binding import Bmgd, FLAG_NO_SLOTS, FLAG_TIMING
     rank, world, local = dist_env()
-    extra_flags = FLAG_BULK_ROWS if args.bulk_rows == 1 else 0
+    extra_flags = 0
     multi = world > 1
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
@@ -268,7 +268,7 @@ def run_ours(args, w):
     host = [inputs.make_buffer(w, k) for k in range(nb)]
     seed0 = w.seed + rank * 1_000_003
     shape = dict(cluster_size=args.cluster_size, ctas_per_chain=args.ctas_per_chain, threads_per_cta=args.threads,
-                 pipeline_depth=args.depth, subpasses_per_stage=args.subpasses)
+                 pipeline_depth=args.depth, subpasses_per_stage=args.subpasses, producer_warps=args.producer_warps)
     sg_per_step = [x.shape[0] * w.T * w.Rc for x, _ in host]
 
     # ---- device-resident measurement

@@ -61,8 +61,6 @@ enum {
                                        assumption under which Eq. (3.1)-(3.3) are derived */
     BMGD_FLAG_NO_SLOTS = 2u,        /* allocate no buffer slots: only bmgd_run_rounds_resident is used */
     BMGD_FLAG_TIMING = 4u,          /* record CUDA events round every launch and copy (bmgd_get_stats) */
-    BMGD_FLAG_BULK_ROWS = 16u,      /* linear/logistic: fetch each row with one bulk copy (cp.async.bulk) instead of
-                                       16-byte cp.async chunks; needs rows that are 16-byte multiples */
     BMGD_FLAG_SOFTMAX_CUDA_CORES = 8u /* softmax: run the two contractions on the CUDA cores, not the tensor cores
                                        (same bf16 inputs; for cross-checking the tensor-core path) */
 };
@@ -87,10 +85,11 @@ typedef struct bmgd_config {
      * (a multiple of cluster_size); the rows of a mini-batch are split among them. */
     int32_t cluster_size;     /* CTAs per thread-block cluster: 1, 2, 4, 8 or 16 */
     int32_t ctas_per_chain;
-    int32_t threads_per_cta;  /* 256, 512 or 1024 */
-    int32_t pipeline_depth;   /* row-prefetch stages held in shared memory: 2, 3 or 4 */
+    int32_t threads_per_cta;  /* threads that compute: a multiple of 32 from 256 to 512 (softmax: 256, 512 or 1024) */
+    int32_t pipeline_depth;   /* row-prefetch stages held in shared memory: 2 to 8 */
     int32_t subpasses_per_stage; /* a stage holds this many sweeps of the CTA over its rows: 1, 2, 4, ... 32 */
-    int32_t reserved[7];      /* must be zero */
+    int32_t producer_warps;   /* linear/logistic: extra warps per CTA that only evaluate the shuffle and fetch rows: 1 to 4 */
+    int32_t reserved[6];      /* must be zero */
 } bmgd_config;
 
 typedef struct bmgd_stats {
@@ -103,7 +102,7 @@ typedef struct bmgd_stats {
     int32_t grid_ctas;         /* shape of the last launch */
     int32_t cluster_size;
     int32_t ctas_per_chain;
-    int32_t threads_per_cta;
+    int32_t threads_per_cta;   /* all warps of a CTA, those that only fetch rows included */
     int32_t pipeline_depth;
     int32_t smem_bytes;
     int32_t chains_in_flight;  /* chains worked on at the same time in the last launch */

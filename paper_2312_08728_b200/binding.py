@@ -25,7 +25,6 @@ FLAG_FIXED_PARTITION = 1
 FLAG_NO_SLOTS = 2
 FLAG_TIMING = 4
 FLAG_SOFTMAX_CUDA_CORES = 8
-FLAG_BULK_ROWS = 16
 
 # every symbol include/bmgd.h declares
 EXPORTS = (
@@ -44,7 +43,8 @@ class BmgdConfig(ctypes.Structure):
         ("compute_stream", ctypes.c_void_p), ("timeout_ms", ctypes.c_double),
         ("cluster_size", ctypes.c_int32), ("ctas_per_chain", ctypes.c_int32),
         ("threads_per_cta", ctypes.c_int32), ("pipeline_depth", ctypes.c_int32),
-        ("subpasses_per_stage", ctypes.c_int32), ("reserved", ctypes.c_int32 * 7),
+        ("subpasses_per_stage", ctypes.c_int32), ("producer_warps", ctypes.c_int32),
+        ("reserved", ctypes.c_int32 * 6),
     ]
 
 
@@ -189,6 +189,7 @@ class Bmgd:
     def __init__(self, N: int, p: int, K: int, loss: int = LOSS_LINEAR, dtype: int = DTYPE_F32, C: int = 1,
                  Rc: int = 1, device: int = 0, flags: int = 0, cluster_size: int = 0, ctas_per_chain: int = 0,
                  threads_per_cta: int = 0, pipeline_depth: int = 0, subpasses_per_stage: int = 0,
+                 producer_warps: int = 0,
                  timeout_ms: float = 0.0,
                  use_torch_stream: bool = False):
         if not torch.cuda.is_available():
@@ -202,6 +203,7 @@ class Bmgd:
         cfg.cluster_size, cfg.ctas_per_chain = cluster_size, ctas_per_chain
         cfg.threads_per_cta, cfg.pipeline_depth, cfg.timeout_ms = threads_per_cta, pipeline_depth, timeout_ms
         cfg.subpasses_per_stage = subpasses_per_stage
+        cfg.producer_warps = producer_warps
         need = ctypes.c_int64()
         self._check(self._lib.bmgd_workspace_bytes(ctypes.byref(cfg), ctypes.byref(need)), "bmgd_workspace_bytes")
         self.device = torch.device("cuda", device)

@@ -110,14 +110,15 @@ int validate(const bmgd_config* c) {
     }
     const int64_t N0 = (c->N + c->K - 1) / c->K;
     if (N0 > 0x7FFFFFFFll) return BMGD_ERR_ARG;
-    for (int i = 0; i < 7; ++i)
+    for (int i = 0; i < 6; ++i)
         if (c->reserved[i] != 0) return BMGD_ERR_ARG;
+    if (c->producer_warps < 0 || c->producer_warps > 4) return BMGD_ERR_ARG;
     if (c->cluster_size != 0 && c->cluster_size != 1 && c->cluster_size != 2 && c->cluster_size != 4 &&
         c->cluster_size != 8 && c->cluster_size != 16)
         return BMGD_ERR_ARG;
-    if (c->threads_per_cta != 0 && c->threads_per_cta != 256 && c->threads_per_cta != 512 && c->threads_per_cta != 1024)
+    if (c->threads_per_cta != 0 && (c->threads_per_cta % 32 != 0 || c->threads_per_cta < 256 || c->threads_per_cta > 1024))
         return BMGD_ERR_ARG;
-    if (c->pipeline_depth != 0 && (c->pipeline_depth < 2 || c->pipeline_depth > 4)) return BMGD_ERR_ARG;
+    if (c->pipeline_depth != 0 && (c->pipeline_depth < 2 || c->pipeline_depth > 8)) return BMGD_ERR_ARG;
     if (c->subpasses_per_stage != 0 && c->subpasses_per_stage != 1 && c->subpasses_per_stage != 2 &&
         c->subpasses_per_stage != 4 && c->subpasses_per_stage != 8 && c->subpasses_per_stage != 16 &&
         c->subpasses_per_stage != 32)
@@ -154,15 +155,17 @@ typedef void (*GlmKernel)(const GlmParams);
 
 struct GlmVariant {
     GlmKernel fn;
-    int vec, lpr, kch, maxt;
+    int vec, lpr, kch, maxc, maxt;
     int cap() const { return vec * lpr * kch; }
-    int max_threads() const { return maxt; }
+    int max_consumer_threads() const { return maxc; }  // warps that compute
+    int max_threads() const { return maxt; }           // consumers plus producers
 };
 
 template <typename T, bool LG>
 const GlmVariant* glm_variants(bool aligned16, int* count) {
     constexpr int V = 16 / (int)sizeof(T);
-#define BMGD_VAR(VEC, LPR, KCH) {bmgdk::glm_kernel<T, VEC, LPR, KCH, LG>, VEC, LPR, KCH, bmgdk::glm_max_threads<T, VEC, KCH>()}
+#define BMGD_VAR(VEC, LPR, KCH) {bmgdk::glm_kernel<T, VEC, LPR, KCH, LG>, VEC, LPR, KCH, \
+                                 bmgdk::glm_max_consumer_threads<T, VEC, KCH>(), bmgdk::glm_max_threads<T, VEC, KCH>()}
     static const GlmVariant wide[] = {BMGD_VAR(V, 8, 1), BMGD_VAR(V, 8, 2), BMGD_VAR(V, 8, 4),
                                       BMGD_VAR(V, 8, 8), BMGD_VAR(V, 16, 8), BMGD_VAR(V, 32, 8)};
     static const GlmVariant narrow[] = {BMGD_VAR(1, 32, 1), BMGD_VAR(1, 32, 2), BMGD_VAR(1, 32, 4), BMGD_VAR(1, 32, 8)};
@@ -190,7 +193,7 @@ int floor_pow2(int v) {
 }
 
 struct LaunchShape {
-    int S, cpc, nteams, threads, depth, passes, rb, smem;
+    int S, cpc, nteams, threads, pwarps, depth, passes, rb, smem;  // threads: of the consumer warps
 };
 
 int max_active_clusters(bmgd* h, GlmKernel fn, int S, int threads, int smem, int* out) {
@@ -214,8 +217,13 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     const int gpw = 32 / var->lpr;
     const int pcap = var->cap();
     LaunchShape L{};
-    L.threads = c.threads_per_cta ? std::min(c.threads_per_cta, var->max_threads())
-                                  : ((c.Rc > 1 && var->max_threads() >= 512) ? 512 : 256);
+    L.threads = c.threads_per_cta ? std::min(c.threads_per_cta, var->max_consumer_threads())
+                                  : ((c.Rc > 1 && var->max_consumer_threads() >= 512) ? 512 : 256);
+    // Producer warps only evaluate the shuffle and issue copies; both are chains of dependent instructions, so several
+    // warps side by side are what keeps them ahead of the consumers.
+    L.pwarps = c.producer_warps ? c.producer_warps : 4;
+    L.pwarps = std::min(L.pwarps, (var->max_threads() - L.threads) / 32);
+    if (L.pwarps < 1) return BMGD_ERR_ARG;
     const int warps = L.threads / 32;
     const int spp = warps * gpw;  // rows a CTA works on at once (one sub-pass)
     const bool pre = var->kch * var->vec <= 16;
@@ -237,7 +245,7 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     // the largest ring we would use (a smaller one can only admit more).
     int max_clusters = 0, fixed_smem = 0, ring_budget = 0;
     for (;;) {
-        fixed_smem = bmgdk::glm_smem_plan(warps, gpw, pre, 1, 0, pcap, eb, S).total_bytes;
+        fixed_smem = bmgdk::glm_smem_plan(warps, gpw, pre, 1, 0, pcap, eb, S, false).total_bytes;
         ring_budget = std::min(h->smem_optin - fixed_smem, 160 * 1024);
         if (ring_budget < 2 * spp * pitch) {  // the per-peer exchange buffers of a large cluster leave no room for rows
             if (c.cluster_size == 0 && S > 1) { S /= 2; continue; }
@@ -248,7 +256,7 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
         BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn, cudaFuncAttributeNonPortableClusterSizeAllowed, S > 8 ? 1 : 0));
         max_clusters = h->sm_count;
         if (S > 1) {
-            int rc = max_active_clusters(h, var->fn, S, L.threads, probe_smem, &max_clusters);
+            int rc = max_active_clusters(h, var->fn, S, L.threads + 32 * L.pwarps, probe_smem, &max_clusters);
             if (rc != BMGD_OK) {
                 if (c.cluster_size == 0 && S > 8) { S = 8; continue; }  // clusters of 16 are optional in hardware
                 return rc;
@@ -278,6 +286,10 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
         L.cpc = cpc;
         L.nteams = std::max(1, std::min(c.Rc, max_clusters / cpc));
     }
+    // a chain that spans clusters keeps only its slice of the peers' packets in shared memory: more room for rows
+    const bool multi = L.cpc > 1;
+    fixed_smem = bmgdk::glm_smem_plan(warps, gpw, pre, 1, 0, pcap, eb, S, multi).total_bytes;
+    ring_budget = std::min(h->smem_optin - fixed_smem, 160 * 1024);
     const int G = L.cpc * S;
     const int rows_per_cta = (n + G - 1) / G;
     const int subpasses = std::max(1, (rows_per_cta + spp - 1) / spp);
@@ -287,17 +299,19 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     const int subpass_bytes = spp * pitch;
     // narrow rows (at most 32 bytes per lane) are swept four sub-passes at a time by the kernel, others two
     int rb = c.subpasses_per_stage ? c.subpasses_per_stage : ((var->kch * 16 <= 32) ? 4 : 2);
-    rb = std::min(rb, var->lpr);
     rb = floor_pow2(std::max(1, std::min(rb, subpasses)));
+    // a producer warp takes at most kMaxBatchesPerProducer batches of 32 row slots per stage
+    while (rb > 1 && rb * spp > 32 * bmgdk::kMaxBatchesPerProducer * L.pwarps) rb /= 2;
+    if (spp > 32 * bmgdk::kMaxBatchesPerProducer * L.pwarps) return BMGD_ERR_ARG;
     while (rb > 1 && 2 * rb * subpass_bytes > ring_budget) rb /= 2;
     L.rb = rb;
     L.passes = (subpasses + rb - 1) / rb;
     const int stage_bytes = rb * subpass_bytes;
-    int depth = c.pipeline_depth ? c.pipeline_depth : 4;  // the kernel keeps 2, 3 or 4 stages in flight
+    int depth = c.pipeline_depth ? c.pipeline_depth : 4;  // ring stages: 2 to 8
     while (depth > 2 && depth * stage_bytes > ring_budget) --depth;
     if (depth * stage_bytes > ring_budget) return BMGD_ERR_UNIMPLEMENTED;
     L.depth = depth;
-    L.smem = bmgdk::glm_smem_plan(warps, gpw, pre, rb, depth, pcap, eb, S).total_bytes;
+    L.smem = bmgdk::glm_smem_plan(warps, gpw, pre, rb, depth, pcap, eb, S, multi).total_bytes;
     (void)rows;
     *out = L;
     return BMGD_OK;
@@ -369,16 +383,16 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
     P.N0 = (uint32_t)rows; P.n = (uint32_t)n; P.M = M; P.T = rounds; P.p = c.p;
     P.Rc = c.Rc; P.S = L.S; P.cpc = L.cpc; P.nteams = L.nteams;
     P.passes = L.passes; P.rb = L.rb; P.depth = L.depth;
+    P.consumer_warps = L.threads / 32; P.producer_warps = L.pwarps;
     P.q_full = (uint32_t)n / (uint32_t)(L.cpc * L.S); P.r_full = (uint32_t)n % (uint32_t)(L.cpc * L.S);
     P.ll_stride = c.p * 2;
     P.tag_base = (uint32_t)h->tag_base;
     P.fixed_partition = (c.flags & BMGD_FLAG_FIXED_PARTITION) ? 1 : 0;
-    P.bulk_rows = (aligned16 && (c.flags & BMGD_FLAG_BULK_ROWS)) ? 1 : 0;
     if ((int64_t)L.nteams * L.cpc > kMaxClustersForExchange) return BMGD_ERR_LAUNCH;
 
     cudaLaunchConfig_t lc{};
     lc.gridDim = dim3((unsigned)(L.nteams * L.cpc * L.S), 1, 1);
-    lc.blockDim = dim3((unsigned)L.threads, 1, 1);
+    lc.blockDim = dim3((unsigned)(L.threads + 32 * L.pwarps), 1, 1);
     lc.dynamicSmemBytes = (size_t)L.smem;
     lc.stream = h->compute;
     cudaLaunchAttribute at[2];
@@ -421,7 +435,7 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
     h->stats.grid_ctas = L.nteams * L.cpc * L.S;
     h->stats.cluster_size = L.S;
     h->stats.ctas_per_chain = L.cpc * L.S;
-    h->stats.threads_per_cta = L.threads;
+    h->stats.threads_per_cta = L.threads + 32 * L.pwarps;
     h->stats.pipeline_depth = L.depth;
     h->stats.subpasses_per_stage = L.rb;
     h->stats.smem_bytes = L.smem;
@@ -800,6 +814,7 @@ int bmgd_run_rounds_noalloc(const void* dev_x, const void* dev_y, int64_t rows, 
     P.N0 = (uint32_t)rows; P.n = (uint32_t)n; P.M = M; P.T = rounds; P.p = p;
     P.Rc = Rc; P.S = L.S; P.cpc = L.cpc; P.nteams = L.nteams;
     P.passes = L.passes; P.rb = L.rb; P.depth = L.depth;
+    P.consumer_warps = L.threads / 32; P.producer_warps = L.pwarps;
     P.q_full = (uint32_t)n / (uint32_t)(L.cpc * L.S); P.r_full = (uint32_t)n % (uint32_t)(L.cpc * L.S);
     P.ll_stride = p * 2;
     P.tag_base = 0;
@@ -807,7 +822,7 @@ int bmgd_run_rounds_noalloc(const void* dev_x, const void* dev_y, int64_t rows, 
 
     cudaLaunchConfig_t lc{};
     lc.gridDim = dim3((unsigned)(L.nteams * L.cpc * L.S), 1, 1);
-    lc.blockDim = dim3((unsigned)L.threads, 1, 1);
+    lc.blockDim = dim3((unsigned)(L.threads + 32 * L.pwarps), 1, 1);
     lc.dynamicSmemBytes = (size_t)L.smem;
     lc.stream = st;
     cudaLaunchAttribute at[2];

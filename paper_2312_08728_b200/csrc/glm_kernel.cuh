@@ -6,26 +6,24 @@
 // replicate chains there are several teams, each taking chains team, team+nteams, ...
 //
 // Per step, in every CTA:
-//   1. rows pi(j) of this CTA's share were prefetched into a shared-memory ring by cp.async,
-//      several stages ahead (rows do not depend on theta, the shuffle is stateless); each lane
-//      evaluates pi for one row and the warp shares the 32 results by shuffle; the copies for a
-//      later stage are issued while the CTA would otherwise wait at a barrier;
-//   2. a group of LPR lanes owns one row: x.theta by an LPR-lane butterfly, the residual
+//   1. rows pi(j) of this CTA's share were fetched into a shared-memory ring by dedicated producer warps
+//      (16-byte cp.async chunks, completion counted on one mbarrier per ring stage), several stages ahead: rows
+//      do not depend on theta and the shuffle is stateless, so the producers run through step, round and chain
+//      boundaries and the evaluation of pi never sits on the path from one theta to the next;
+//   2. in the consumer warps a group of LPR lanes owns one row: x.theta by an LPR-lane butterfly, the residual
 //      (x.theta - y, or sigmoid(x.theta) - y), then g += r * x with x still in registers, so a
 //      row is read from HBM once and from shared memory once;
-//   3. the group partials are summed in fixed order (shuffles, then shared memory).  With one
-//      cluster per chain every CTA pushes its partial to every peer through distributed shared
-//      memory and one cluster barrier follows.  With several clusters the partials are
-//      reduce-scattered inside the cluster (CTA r owns a slice of the predictors), the slice sums
-//      cross clusters as tagged 8-byte packets in global memory (value and step tag travel in one
-//      64-bit store, so a reader needs no separate flag or fence; only the slice owner polls), and
-//      the totals are pushed back to every peer before a second cluster barrier;
+//   3. the group partials are summed in fixed order (shuffles, then shared memory).  With one cluster per chain
+//      every CTA pushes its partial sums into the shared memory of every peer as tagged 8-byte packets (value and
+//      step tag travel in one 64-bit store, so a reader needs no separate flag, fence or barrier) and sums the
+//      packets that arrive in its own.  With several clusters the partials are reduce-scattered inside the
+//      cluster the same way (CTA r owns a slice of the predictors), the slice sums cross clusters as tagged
+//      packets in global memory (only the slice owner polls), and the totals are pushed to every peer;
 //   4. every CTA applies theta <- theta - (alpha/n_m) g to its own register copy of theta.
 // All sums have a fixed order, so all CTAs hold bit-identical theta and runs are reproducible.
 //
-// Every wait on another CTA is bounded: when the budget runs out the kernel records
-// BMGD_ERR_TIMEOUT in the status word, stops waiting for the rest of the launch (barriers stay
-// matched) and returns.
+// Every wait on another warp or CTA is bounded: when the budget runs out the kernel records
+// BMGD_ERR_TIMEOUT in the status word, stops waiting for the rest of the launch and returns.
 #pragma once
 #include <cstdint>
 #include <cuda_runtime.h>
@@ -35,6 +33,8 @@
 namespace bmgdk {
 
 constexpr int kMaxCpc = 20;        // clusters per chain the packet exchange is unrolled for
+constexpr int kMaxClusterSize = 16; // CTAs per cluster
+constexpr int kMaxBatchesPerProducer = 2;  // batches of 32 row slots one producer warp takes in one ring stage
 constexpr int kStatusTimeout = -5; // == BMGD_ERR_TIMEOUT
 
 struct GlmParams {
@@ -56,14 +56,15 @@ struct GlmParams {
     int S;                // cluster size
     int cpc;              // clusters per chain
     int nteams;
+    int consumer_warps;   // warps that compute (at least 8)
+    int producer_warps;   // warps that fetch rows
     int passes;           // ring stages per step
-    int rb;               // sub-passes per ring stage (a power of two, at most LPR)
-    int depth;            // ring stages in flight: 2, 3 or 4
+    int rb;               // sub-passes per ring stage
+    int depth;            // ring stages: 2 to 8
     uint32_t q_full, r_full;  // n / G and n % G: how a full mini-batch is dealt to the G CTAs
     int ll_stride;        // packets per cluster slot
     uint32_t tag_base;
     int fixed_partition;
-    int bulk_rows;        // rows travel as one bulk copy each (cp.async.bulk) instead of 16-byte cp.async chunks
 };
 
 // ---------------------------------------------------------------- small PTX wrappers
@@ -78,33 +79,17 @@ __device__ __forceinline__ void cp_async(uint32_t dst_smem, const void* src) {
         asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst_smem), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-// cp.async.wait_group takes an immediate: the ring is 2, 3 or 4 stages deep.
-__device__ __forceinline__ void cp_async_wait_ring(int depth) {
-    if (depth == 4) asm volatile("cp.async.wait_group 3;" ::: "memory");
-    else if (depth == 3) asm volatile("cp.async.wait_group 2;" ::: "memory");
-    else asm volatile("cp.async.wait_group 1;" ::: "memory");
-}
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
-
-// One predicated copy chunk at a constant byte offset from both addresses.
-template <int BYTES, int OFF>
-__device__ __forceinline__ void cp_async_at(uint32_t dst_smem, const void* src, uint32_t pred) {
+// One chunk of BYTES bytes: copied from `src` if `have`, otherwise written as zeros (nothing is read from `src`).
+template <int BYTES>
+__device__ __forceinline__ void cp_async_fill(uint32_t dst_smem, const void* src, bool have) {
+    const uint32_t n = have ? (uint32_t)BYTES : 0u;
     if constexpr (BYTES == 16)
-        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %2, 0;\n\t@p cp.async.cg.shared.global [%0+%3], [%1+%3], 16;\n\t}"
-                     ::"r"(dst_smem), "l"(src), "r"(pred), "n"(OFF) : "memory");
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "r"(n) : "memory");
     else if constexpr (BYTES == 8)
-        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %2, 0;\n\t@p cp.async.ca.shared.global [%0+%3], [%1+%3], 8;\n\t}"
-                     ::"r"(dst_smem), "l"(src), "r"(pred), "n"(OFF) : "memory");
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst_smem), "l"(src), "r"(n) : "memory");
     else
-        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %2, 0;\n\t@p cp.async.ca.shared.global [%0+%3], [%1+%3], 4;\n\t}"
-                     ::"r"(dst_smem), "l"(src), "r"(pred), "n"(OFF) : "memory");
-}
-template <int BYTES, int STRIDE, int K, int KCH>
-__device__ __forceinline__ void cp_async_chunks(uint32_t dst_smem, const void* src, uint32_t kmask) {
-    if constexpr (K < KCH) {
-        cp_async_at<BYTES, K * STRIDE>(dst_smem, src, kmask & (1u << K));
-        cp_async_chunks<BYTES, STRIDE, K + 1, KCH>(dst_smem, src, kmask);
-    }
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst_smem), "l"(src), "r"(n) : "memory");
 }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -127,6 +112,15 @@ __device__ __forceinline__ void st_shared_zero16(uint32_t addr) {
 __device__ __forceinline__ void st_cluster(uint32_t addr, double v) {
     asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(addr), "d"(v) : "memory");
 }
+// A 64-bit store into a peer's shared memory and a re-read of one's own: value and tag travel together.
+__device__ __forceinline__ void st_cluster_u64(uint32_t addr, unsigned long long v) {
+    asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(addr), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_shared_volatile_u64(uint32_t addr) {
+    unsigned long long v;
+    asm volatile("ld.volatile.shared.u64 %0, [%1];" : "=l"(v) : "r"(addr) : "memory");
+    return v;
+}
 __device__ __forceinline__ void cluster_arrive_release() {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
 }
@@ -140,6 +134,14 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// one row, global -> shared, completion counted in bytes on `bar`; addresses and size are 16-byte multiples
+__device__ __forceinline__ void bulk_copy_row(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 // the arrival happens once every cp.async this thread has issued so far has landed
 __device__ __forceinline__ void mbar_arrive_after_copies(uint32_t bar) {
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
@@ -151,12 +153,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
-// generic-proxy writes to shared memory become ordered with the bulk copies' writes and the tensor core's reads
+// generic-proxy writes to shared memory become ordered with bulk copies into, and tensor-core reads of, the same bytes
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-// one row, global -> shared, completion counted in bytes on `bar`; addresses and size are 16-byte multiples
-__device__ __forceinline__ void bulk_copy_row(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+// a barrier among the consumer warps only (the producer warps never join it)
+__device__ __forceinline__ void consumer_sync(int consumer_threads) {
+    asm volatile("bar.sync 1, %0;" ::"r"(consumer_threads) : "memory");
 }
 
 __device__ __forceinline__ void st_packet(unsigned long long* p, unsigned long long v) {
@@ -201,22 +202,28 @@ struct GlmSmemPlan {
     int warp_stage_bytes;  // one warp's share of one ring stage
     int ring_off, ring_bytes;
     int gpart_rows;        // partial-gradient rows summed per CTA
-    int gpart_off, cpart_off, gfin_off;
+    int gpart_off, gfin_off;
+    int cpk_off, cpk_stride;  // tagged packets from the cluster's CTAs: [2][S][cpk_stride] 64-bit words
+    int gpk_off;              // tagged packets carrying the totals (several clusters per chain): [2][pcap * words]
     int total_bytes;
 };
 
+// `multi`: a chain spans several clusters, so a CTA receives only its slice of the predictors from its peers.
 __host__ __device__ inline GlmSmemPlan glm_smem_plan(int warps, int gpw, bool prereduce, int rb, int depth, int pcap,
-                                                     int elem_bytes, int S) {
+                                                     int elem_bytes, int S, bool multi) {
     GlmSmemPlan s;
+    const int words = elem_bytes / 4;
     s.pitch = pcap * elem_bytes + 16;
     s.warp_stage_bytes = rb * gpw * s.pitch;
     s.ring_off = 1024;  // room for one mbarrier per (warp, stage) in front of the ring
     s.ring_bytes = warps * depth * s.warp_stage_bytes;
     s.gpart_rows = prereduce ? warps : warps * gpw;
     s.gpart_off = s.ring_off + s.ring_bytes;
-    s.cpart_off = s.gpart_off + s.gpart_rows * pcap * elem_bytes;
-    s.gfin_off = s.cpart_off + 2 * S * pcap * elem_bytes;
-    s.total_bytes = s.gfin_off + pcap * elem_bytes;
+    s.gfin_off = s.gpart_off + s.gpart_rows * pcap * elem_bytes;
+    s.cpk_off = s.gfin_off + pcap * elem_bytes;
+    s.cpk_stride = (multi ? (pcap + S - 1) / S : pcap) * words;
+    s.gpk_off = s.cpk_off + (S > 1 ? 2 * S * s.cpk_stride * 8 : 0);
+    s.total_bytes = s.gpk_off + ((multi && S > 1) ? 2 * pcap * words * 8 : 0);
     return s;
 }
 
@@ -238,10 +245,18 @@ __device__ long long g_trace[kTraceSteps * kTracePhases];
 
 // ---------------------------------------------------------------- the kernel
 
-// Largest CTA a variant is compiled for: wide per-lane state (or fp64) needs the 255-register budget.
+// Consumer warps a variant can run with, and the largest CTA it is compiled for (consumers plus producers): wide
+// per-lane state (or fp64) needs a large register budget per thread.
+template <typename T, int VEC, int KCH>
+__host__ __device__ constexpr int glm_max_consumer_threads() {
+    return (sizeof(T) == 8 || KCH * VEC >= 32) ? 256 : 512;
+}
+#ifndef BMGD_GLM_MAX_THREADS
+#define BMGD_GLM_MAX_THREADS 640
+#endif
 template <typename T, int VEC, int KCH>
 __host__ __device__ constexpr int glm_max_threads() {
-    return (sizeof(T) == 8 || KCH * VEC >= 32) ? 256 : 512;
+    return (sizeof(T) == 8 || KCH * VEC >= 32) ? 256 + 128 : BMGD_GLM_MAX_THREADS;  // registers come in units of four warps
 }
 // Few values per lane: fold the row groups of a warp together by shuffles before shared memory.
 template <int VEC, int KCH>
@@ -250,12 +265,11 @@ __host__ __device__ constexpr bool glm_prereduce() {
 }
 
 // How mini-batch rows [lo, lo+nm) are dealt to CTA g of G: a contiguous run of `cnt` rows from lo+a.
-// nsp is the number of sub-passes of the step in which the calling warp has at least one row.
 struct RowShare {
-    uint32_t lo, a, cnt, nsp;
+    uint32_t lo, a, cnt;
 };
 __device__ __forceinline__ RowShare row_share(uint32_t m, uint32_t n, uint32_t N0, uint32_t g, uint32_t G,
-                                              uint32_t q_full, uint32_t r_full, uint32_t warp_first, int spp_log2) {
+                                              uint32_t q_full, uint32_t r_full) {
     RowShare s;
     s.lo = m * n;
     const uint32_t nm = min(n, N0 - s.lo);
@@ -263,7 +277,83 @@ __device__ __forceinline__ RowShare row_share(uint32_t m, uint32_t n, uint32_t N
     if (nm != n) { q = nm / G; r = nm % G; }
     s.a = g * q + min(g, r);
     s.cnt = q + (g < r ? 1u : 0u);
-    s.nsp = (s.cnt > warp_first) ? ((s.cnt - warp_first - 1u) >> spp_log2) + 1u : 0u;
+    return s;
+}
+
+// Two indices through the shuffle at once, each under its own round keys: the two Feistel chains are independent,
+// so their latencies overlap.
+__device__ __forceinline__ void perm_index2(uint32_t& x0, const RoundKeys& k0, uint32_t& x1, const RoundKeys& k1,
+                                            const FeistelDomain& d) {
+    bool w0 = true, w1 = true;  // still walking the cycle
+    do {
+        uint32_t L0 = x0 >> d.c, R0 = x0 & d.maskC;
+        uint32_t L1 = x1 >> d.c, R1 = x1 & d.maskC;
+#pragma unroll
+        for (int r = 0; r < 8; r += 2) {
+            L0 ^= feistel_f(R0, k0.k[r]) & d.maskA;
+            L1 ^= feistel_f(R1, k1.k[r]) & d.maskA;
+            R0 ^= feistel_f(L0, k0.k[r + 1]) & d.maskC;
+            R1 ^= feistel_f(L1, k1.k[r + 1]) & d.maskC;
+        }
+        if (w0) { x0 = (L0 << d.c) | R0; w0 = x0 >= d.N0; }
+        if (w1) { x1 = (L1 << d.c) | R1; w1 = x1 >= d.N0; }
+    } while (w0 || w1);
+}
+
+// Reads `count` tagged packets (NW 64-bit words each: value word in the low half, step tag in the high half) through
+// `load(k, w)` until every tag equals `tag`, then returns the sum of the values in the order k = 0, 1, ....  Packets
+// are taken CH at a time: all loads of a sweep over a chunk are issued before the first tag is checked.  The wait is
+// bounded: when the budget runs out, or another thread has given up, the error is recorded, `aborted` is set and the
+// result is void.
+template <typename T, int MAXK, int CH, typename Load>
+__device__ __forceinline__ T gather_packets(int count, uint32_t tag, bool& aborted, const GlmParams& P, Load load) {
+    constexpr int NW = Words<T>::N;
+    T s = T(0);
+#pragma unroll
+    for (int k0 = 0; k0 < MAXK; k0 += CH) {
+        if (k0 >= count) break;
+        unsigned long long v[CH][NW];
+        unsigned long long t0 = 0;
+        uint32_t spins = 0;
+        while (!aborted) {
+#pragma unroll
+            for (int k = 0; k < CH; ++k) {
+                if (k0 + k < count) {
+#pragma unroll
+                    for (int w = 0; w < NW; ++w) v[k][w] = load(k0 + k, w);
+                }
+            }
+            bool ok = true;
+#pragma unroll
+            for (int k = 0; k < CH; ++k) {
+                if (k0 + k < count) {
+#pragma unroll
+                    for (int w = 0; w < NW; ++w) ok &= ((uint32_t)(v[k][w] >> 32) == tag);
+                }
+            }
+            if (ok) break;
+            if ((++spins & 0x3FFu) == 0u) {
+                const unsigned long long now = global_ns();
+                if (t0 == 0) t0 = now;
+                if (now - t0 > P.timeout_ns || ((volatile int*)P.status)[1] != 0) {
+                    atomicCAS(P.status, 0, kStatusTimeout);
+                    atomicExch(P.status + 1, 1);
+                    aborted = true;
+                }
+            }
+        }
+        if (!aborted) {
+#pragma unroll
+            for (int k = 0; k < CH; ++k) {
+                if (k0 + k < count) {
+                    uint32_t w32[NW];
+#pragma unroll
+                    for (int w = 0; w < NW; ++w) w32[w] = (uint32_t)v[k][w];
+                    s += Words<T>::make(w32);
+                }
+            }
+        }
+    }
     return s;
 }
 
@@ -322,21 +412,40 @@ __device__ __forceinline__ void row_step(const unsigned char* rowp, int y_rel, c
     for (int i = 0; i < NV; ++i) gacc[i] = fma(res, x[i], gacc[i]);
 }
 
+// Waits for a phase of an mbarrier in this CTA's shared memory with the kernel's bounded-wait protocol.
+__device__ __forceinline__ void bounded_mbar_wait(uint32_t bar, uint32_t parity, bool& aborted, const GlmParams& P) {
+    unsigned long long t0 = 0;
+    uint32_t spins = 0;
+    while (!aborted && !mbar_try_wait(bar, parity)) {
+        if ((++spins & 0x3Fu) == 0u) {
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > P.timeout_ns || ((volatile int*)P.status)[1] != 0) {
+                atomicCAS(P.status, 0, kStatusTimeout);
+                atomicExch(P.status + 1, 1);
+                aborted = true;
+            }
+        }
+    }
+}
+
 // T: float or double.  VEC: elements per copy chunk (16 bytes worth, or 1 when rows are not
 // 16-byte multiples).  LPR: lanes per row.  KCH: chunks per lane.  A row has at most
 // PCAP = LPR*KCH*VEC predictors.  LOGISTIC: sigmoid residual instead of the linear one.
 //
-// Row slots of a CTA within one step are numbered u = (sp*W + warp)*GPW + grp, sp = sub-pass:
-// in sub-pass sp every warp works on GPW rows at once.  A ring stage holds `rb` sub-passes.
-// A ring row is PCAP values wide whatever p is; the part beyond p is zeroed once and never written,
-// and a slot without a row is zero-filled, so the inner loop carries no predicates.
-// blockDim.x is 256, 512 or 1024.
+// A CTA has P.consumer_warps warps that compute and P.producer_warps warps that only fetch rows.
+// Row slots of a CTA within one step are numbered u = (sp*W + warp)*GPW + grp, sp = sub-pass: in sub-pass sp
+// consumer warp `warp` works on GPW rows at once.  A ring stage holds `rb` sub-passes, i.e. R = rb*W*GPW
+// consecutive slots, laid out in this order with a pitch of PCAP values plus 16 bytes for y; the part of a ring
+// row beyond p is zeroed once and never written, and a slot without a row is zero-filled by its copy, so the
+// inner loop carries no predicates.  Each stage has a "full" mbarrier (the producers' copies have landed) and an
+// "empty" one (every consumer warp has read it).
 template <typename T, int VEC, int LPR, int KCH, bool LOGISTIC>
 __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(const GlmParams P) {
     constexpr int GPW = 32 / LPR;            // row groups per warp
     constexpr int NV = KCH * VEC;            // values per lane
     constexpr int PCAP = LPR * KCH * VEC;    // predictor capacity
-    constexpr int FPT = (PCAP + 255) / 256;  // features per thread in the reductions (blockDim >= 256)
+    constexpr int FPT = (PCAP + 255) / 256;  // features per thread in the reductions (at least 256 consumer threads)
     constexpr int CB = VEC * (int)sizeof(T); // copy chunk bytes
     constexpr int NW = Words<T>::N;
     constexpr bool PRE = glm_prereduce<VEC, KCH>();
@@ -345,48 +454,35 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
 
     extern __shared__ __align__(16) unsigned char smem[];
 
-    const int tid = threadIdx.x, nthreads = blockDim.x;
-    const int W = nthreads >> 5, warp = tid >> 5, lane = tid & 31;
-    const int grp = lane / LPR, sub = lane % LPR;
+    const int tid = threadIdx.x;
+    const int W = P.consumer_warps, NPW = P.producer_warps;  // blockDim.x == 32 * (W + NPW)
+    const int nthreads = W * 32;                             // consumer threads: the ones that reduce and exchange
+    const int warp = tid >> 5, lane = tid & 31;
     const int S = P.S, cpc = P.cpc, G = cpc * S;
     const int rank = (S > 1) ? (int)cluster_ctarank() : 0;
     const int cluster_id = blockIdx.x / S;
     const int team = cluster_id / cpc, kc = cluster_id % cpc;
     const int g = kc * S + rank;
-    const int p = P.p, nchunks = p / VEC;
+    const int p = P.p;
     const uint32_t N0 = P.N0, n = P.n, M = P.M;
     const int T_rounds = P.T, passes = P.passes, RB = P.rb, D = P.depth;
-    const int spp_log2 = 31 - __clz(W * GPW);          // rows per sub-pass is a power of two
-    const uint32_t warp_first = (uint32_t)(warp * GPW); // first row slot of this warp in sub-pass 0
+    const int spp = W * GPW;  // rows the CTA works on at once (one sub-pass)
 
-    const GlmSmemPlan plan = glm_smem_plan(W, GPW, PRE, RB, D, PCAP, (int)sizeof(T), S);
+    const GlmSmemPlan plan = glm_smem_plan(W, GPW, PRE, RB, D, PCAP, (int)sizeof(T), S, cpc > 1);
     const int pitch = plan.pitch;
-    unsigned char* my_ring = smem + plan.ring_off + warp * D * plan.warp_stage_bytes;
-    const uint32_t my_bars = smem_u32(smem) + (uint32_t)(warp * D * 8);  // one mbarrier per stage of this warp's ring
-    const bool bulk = P.bulk_rows != 0;
-    T* gpart = reinterpret_cast<T*>(smem + plan.gpart_off);
-    T* cpart = reinterpret_cast<T*>(smem + plan.cpart_off);
-    T* gfin = reinterpret_cast<T*>(smem + plan.gfin_off);
-    const int lane_off = grp * pitch + sub * CB;  // this lane's first chunk inside a sub-pass of its warp
-    const int subpass_bytes = GPW * pitch;
-    const int y_rel = YOFF - sub * CB;
-
-    const unsigned char* Xb = static_cast<const unsigned char*>(P.X) + sub * CB;
-    const T* yb = static_cast<const T*>(P.y);
-    const uint32_t row_bytes = (uint32_t)p * (uint32_t)sizeof(T);
-    const FeistelDomain dom = make_domain(N0);
-    const int slice = (p + S - 1) / S;  // predictors owned by one CTA of a cluster in the sliced exchange
-    uint32_t kmask = 0;                 // chunk k of this lane lies inside the row
-#pragma unroll
-    for (int k = 0; k < KCH; ++k) kmask |= (sub + k * LPR < nchunks) ? (1u << k) : 0u;
-    const T scale_full = (T)P.scale_full, scale_last = (T)P.scale_last;
-
+    const int stage_bytes = W * plan.warp_stage_bytes;
+    const uint32_t full_bars = smem_u32(smem), empty_bars = smem_u32(smem) + 128u;  // one 8-byte mbarrier per stage each
     const int nch = (team < P.Rc) ? (P.Rc - team + P.nteams - 1) / P.nteams : 0;
-    uint32_t to_issue = (uint32_t)nch * (uint32_t)T_rounds * M * (uint32_t)passes;  // the host keeps this below 2^32
+    const uint32_t total_stages = (uint32_t)nch * (uint32_t)T_rounds * M * (uint32_t)passes;  // the host keeps this below 2^32
 
-    // zero all of shared memory once: row tails beyond p and never-written slots must read as zero
-    for (int i = plan.ring_off + tid * 16; i < plan.total_bytes; i += nthreads * 16) st_shared_zero16(smem_u32(smem + i));
-    if (tid < W * D) mbar_init(smem_u32(smem) + (uint32_t)(tid * 8), 33u);  // 32 lanes after their copies + the byte count
+    // zero all of shared memory once: row tails beyond p and packet tags must read as zero
+    for (int i = plan.ring_off + tid * 16; i < plan.total_bytes; i += (int)blockDim.x * 16) st_shared_zero16(smem_u32(smem + i));
+    if (tid < D) {
+        // every producer lane, once its element copies have landed; with bulk row copies, also one lane per producer
+        // warp announcing that warp's byte count
+        mbar_init(full_bars + (uint32_t)(tid * 8), (uint32_t)(NPW * (CB == 16 ? 33 : 32)));
+        mbar_init(empty_bars + (uint32_t)(tid * 8), (uint32_t)W);           // one lane of every consumer warp
+    }
     fence_barrier_init();
     fence_async_proxy();  // bulk copies will overwrite bytes zeroed here
     __syncthreads();
@@ -395,354 +491,414 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
         cluster_wait_acquire();
     }
 
-    // ---- prefetch cursor: runs D stages ahead of the compute cursor
-    int pf_ci = 0, pf_t = 0, pf_sidx = 0, pf_slot = 0;
-    uint32_t pf_m = 0;
-    uint32_t pf_rows = kNoRow;  // this lane's row of the current batch of 32 row slots
-    RoundKeys pfk = round_keys(P.seed, (uint32_t)team, 0u);
-    RowShare pfs = row_share(0u, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full, warp_first, spp_log2);
-
-    auto issue_one = [&]() {
-        if (to_issue != 0u) {
-            --to_issue;
-            uint32_t dst = smem_u32(my_ring + pf_slot * plan.warp_stage_bytes) + lane_off;
-            const uint32_t pf_bar = my_bars + (uint32_t)(pf_slot * 8);
-            int pf_rows_in_stage = 0;
-            int sp = pf_sidx * RB;
-            for (int r = 0; r < RB; ++r, ++sp, dst += subpass_bytes) {
-                const int bi = sp & (LPR - 1);
-                if (bi == 0) {  // a new batch: lane l takes sub-pass sp + l/GPW, group l%GPW
-                    const uint32_t u = (((uint32_t)(sp + lane / GPW)) << spp_log2) + warp_first + (lane % GPW);
-                    pf_rows = (u < pfs.cnt) ? perm_index(pfs.lo + pfs.a + u, dom, pfk) : kNoRow;
-                }
-                if ((uint32_t)sp < pfs.nsp) {  // otherwise the whole warp skips this sub-pass, here and in the compute loop
-                    const uint32_t row = __shfl_sync(0xFFFFFFFFu, pf_rows, bi * GPW + grp);
-                    if (row != kNoRow) {
-                        if (bulk) {
-                            if (sub == 0) {  // one bulk copy per row; its bytes are counted on the stage's mbarrier
-                                bulk_copy_row(dst, Xb + (size_t)row * row_bytes, row_bytes, pf_bar);
-                                cp_async<(int)sizeof(T)>(dst + YOFF, yb + row);
-                            }
-                        } else {
-                            cp_async_chunks<CB, LPR * CB, 0, KCH>(dst, Xb + (size_t)row * row_bytes, kmask);
-                            cp_async_at<(int)sizeof(T), 0>(dst + y_rel, yb + row, sub == 0 ? 1u : 0u);
-                        }
-                    } else {  // no row for this slot: it must contribute nothing
-#pragma unroll
-                        for (int k = 0; k < KCH; ++k) {
-                            if constexpr (CB == 16) st_shared_zero16(dst + k * LPR * CB);
-                            else if constexpr (CB == 8) asm volatile("st.shared.b64 [%0], %1;" ::"r"(dst + k * LPR * CB), "l"(0ull) : "memory");
-                            else asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst + k * LPR * CB), "r"(0) : "memory");
-                        }
-                        if (sub == 0) st_shared_zero16(dst + y_rel);
-                        if (bulk) fence_async_proxy();  // a later bulk copy will overwrite these bytes
-                    }
-                    if (bulk) pf_rows_in_stage += __popc(__ballot_sync(0xFFFFFFFFu, row != kNoRow && sub == 0));
-                }
-            }
-            if (++pf_sidx == passes) {
-                pf_sidx = 0;
-                if (++pf_m == M) {
-                    pf_m = 0;
-                    if (++pf_t == T_rounds) { pf_t = 0; ++pf_ci; }
-                    if (pf_ci < nch)
-                        pfk = round_keys(P.seed, (uint32_t)(team + pf_ci * P.nteams),
-                                         P.fixed_partition ? 0u : (uint32_t)pf_t);
-                }
-                pfs = row_share(pf_m, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full, warp_first, spp_log2);
-            }
-            if (bulk) {
-                if (lane == 0) mbar_arrive_expect_tx(pf_bar, (uint32_t)pf_rows_in_stage * row_bytes);
-                mbar_arrive_after_copies(pf_bar);
-            }
-            if (++pf_slot == D) pf_slot = 0;
-        }
-        if (!bulk) cp_async_commit();
-        __syncwarp();  // lanes walked the cycle for different lengths: meet again before any aligned barrier
-    };
-
-    for (int s = 0; s < D; ++s) issue_one();
-
-    int cs_slot = 0;         // ring slot the compute cursor reads next
-    uint32_t cs_phase = 0;   // parity of that slot's mbarrier phase (bulk-copy mode)
-    uint32_t step_count = 0; // steps this team has finished in this launch
     bool aborted = false;
 
-    for (int ci = 0; ci < nch; ++ci) {
-        const int chain = team + ci * P.nteams;
-        T* theta_g = static_cast<T*>(P.theta) + (size_t)chain * p;
+    if (warp >= W) {
+        // ================================================================ producer warps
+        // Rows do not depend on theta and the shuffle is stateless, so the producers run up to D stages ahead of
+        // the consumers, through mini-batch, round and chain boundaries.  Slots of a stage are taken 32 at a time
+        // (a batch; ownership of batches rotates over the producer warps): lane l evaluates pi for slot 32b + l and
+        // fetches that row, with one bulk copy when rows are 16-byte multiples.  Two consecutive stages are worked on
+        // together, so that their two shuffle evaluations overlap.
+        const int pw = warp - W;
+        const int R = RB * spp;
+        const int nbatch = (R + 31) >> 5;
+        const int nchunks = p / VEC;
+        int lpr_c = 1;  // lanes that copy one row: the power of two at or above nchunks, at most 32
+        while (lpr_c < nchunks && lpr_c < 32) lpr_c <<= 1;
+        const int rpi = 32 / lpr_c;                        // rows per copy iteration
+        const int cpl = (nchunks + lpr_c - 1) / lpr_c;     // chunks per lane and row
+        const int rsub = lane / lpr_c, cl = lane % lpr_c;
+        const unsigned char* Xrows = static_cast<const unsigned char*>(P.X);
+        const unsigned char* Xb = Xrows + (size_t)cl * CB;
+        const T* yb = static_cast<const T*>(P.y);
+        const uint32_t row_bytes = (uint32_t)p * (uint32_t)sizeof(T);
+        const FeistelDomain dom = make_domain(N0);
+        const uint32_t ring_base = smem_u32(smem + plan.ring_off);
 
-        T th[NV];
-#pragma unroll
-        for (int k = 0; k < KCH; ++k) {
-            const int c = sub + k * LPR;
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) th[k * VEC + e] = (c < nchunks) ? theta_g[c * VEC + e] : T(0);
-        }
-
-        for (int t = 0; t < T_rounds; ++t) {
-            for (uint32_t m = 0; m < M; ++m) {
-                const RowShare sh = row_share(m, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full, warp_first, spp_log2);
-                BMGD_STAMP(0);
-
-                T gacc[NV];
-#pragma unroll
-                for (int i = 0; i < NV; ++i) gacc[i] = T(0);
-
-                int sp_left = (int)sh.nsp;  // sub-passes of this step in which the warp still has rows
-                for (int sidx = 0; sidx < passes; ++sidx) {
-                    if (bulk) {  // bounded wait on this warp's stage barrier
-                        const uint32_t bar = my_bars + (uint32_t)(cs_slot * 8);
-                        unsigned long long t0 = 0;
-                        uint32_t spins = 0;
-                        while (!aborted && !mbar_try_wait(bar, cs_phase)) {
-                            if ((++spins & 0x3Fu) == 0u) {
-                                const unsigned long long now = global_ns();
-                                if (t0 == 0) t0 = now;
-                                if (now - t0 > P.timeout_ns || ((volatile int*)P.status)[1] != 0) {
-                                    atomicCAS(P.status, 0, kStatusTimeout);
-                                    atomicExch(P.status + 1, 1);
-                                    aborted = true;
-                                }
-                            }
-                        }
-                    } else {
-                        cp_async_wait_ring(D);
-                    }
-                    __syncwarp();
-                    const unsigned char* rowp = my_ring + cs_slot * plan.warp_stage_bytes + lane_off;
-                    if (++cs_slot == D) { cs_slot = 0; cs_phase ^= 1u; }
-                    int nsub = min(sp_left, RB);
-                    sp_left -= nsub;
-                    if constexpr (NV * (int)sizeof(T) <= 32) {  // narrow rows: four independent rows in flight per group
-                        for (; nsub >= 4; nsub -= 4, rowp += 4 * subpass_bytes) {
-                            row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, y_rel, th, gacc);
-                            row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + subpass_bytes, y_rel, th, gacc);
-                            row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + 2 * subpass_bytes, y_rel, th, gacc);
-                            row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + 3 * subpass_bytes, y_rel, th, gacc);
-                        }
-                    }
-                    for (; nsub >= 2; nsub -= 2, rowp += 2 * subpass_bytes) {  // two independent rows in flight per group
-                        row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, y_rel, th, gacc);
-                        row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + subpass_bytes, y_rel, th, gacc);
-                    }
-                    if (nsub) row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, y_rel, th, gacc);
-                    if (sidx + 1 < passes) {  // refill the slot just read; the last one of a step waits for a barrier
-                        __syncwarp();
-                        issue_one();
-                    }
+        struct Cursor {  // which stage comes next, and what it needs
+            int ci, t, sidx;
+            uint32_t m;
+            RoundKeys rk;
+            RowShare sh;
+        };
+        Cursor cur;
+        cur.ci = 0; cur.t = 0; cur.sidx = 0; cur.m = 0u;
+        cur.rk = round_keys(P.seed, (uint32_t)team, 0u);
+        cur.sh = row_share(0u, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full);
+        auto advance = [&](Cursor& c) {
+            if (++c.sidx == passes) {
+                c.sidx = 0;
+                if (++c.m == M) {
+                    c.m = 0;
+                    if (++c.t == T_rounds) { c.t = 0; ++c.ci; }
+                    if (c.ci < nch)
+                        c.rk = round_keys(P.seed, (uint32_t)(team + c.ci * P.nteams), P.fixed_partition ? 0u : (uint32_t)c.t);
                 }
-                BMGD_STAMP(1);
+                c.sh = row_share(c.m, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full);
+            }
+        };
+        int slot = 0;
+        uint32_t empty_parity = 1u;  // a fresh mbarrier lets a wait on parity 1 through
 
-                // ---- sum the partial gradients of this CTA in fixed order
-                if constexpr (PRE) {
-#pragma unroll
-                    for (int off = LPR; off < 32; off <<= 1)
-#pragma unroll
-                        for (int i = 0; i < NV; ++i) gacc[i] += __shfl_xor_sync(0xFFFFFFFFu, gacc[i], off);
+        // Copies the batch whose first slot is s0; lane l holds the row of slot s0 + l (kNoRow: the slot stays empty).
+        // Rows that are 16-byte multiples travel as one bulk copy each, counted in bytes on the stage's barrier (the
+        // return value is the number of rows this warp sent that way); others go element by element.
+        auto copy_batch = [&](uint32_t stage_base, uint32_t full_bar, int s0, uint32_t rows) -> uint32_t {
+            const int left = R - s0;  // slots of this batch that exist
+            if constexpr (CB == 16) {
+                const bool have = lane < left && rows != kNoRow;
+                const uint32_t dst = stage_base + (uint32_t)((s0 + lane) * pitch);
+                if (have) {
+                    bulk_copy_row(dst, Xrows + (size_t)rows * row_bytes, row_bytes, full_bar);
+                    cp_async_fill<(int)sizeof(T)>(dst + YOFF, yb + rows, true);
+                } else if (lane < left) {  // no row for this slot: it must contribute nothing
+                    for (int k = 0; k < nchunks; ++k) st_shared_zero16(dst + (uint32_t)(k * 16));
+                    st_shared_zero16(dst + YOFF);
+                    fence_async_proxy();  // a later bulk copy will overwrite these bytes
                 }
-                if (!PRE || grp == 0) {
-                    T* gp = gpart + (PRE ? warp : warp * GPW + grp) * PCAP + sub * VEC;
-#pragma unroll
-                    for (int k = 0; k < KCH; ++k) {
-                        if constexpr (CB == 16 && sizeof(T) == 4)
-                            *reinterpret_cast<float4*>(gp + k * LPR * VEC) =
-                                make_float4(gacc[k * VEC], gacc[k * VEC + 1], gacc[k * VEC + 2], gacc[k * VEC + 3]);
-                        else if constexpr (CB == 16)
-                            *reinterpret_cast<double2*>(gp + k * LPR * VEC) = make_double2(gacc[k * VEC], gacc[k * VEC + 1]);
-                        else
-                            gp[k * LPR] = gacc[k];
-                    }
-                }
-                if (S == 1 && cpc == 1) {
-                    __syncwarp();
-                    issue_one();
-                }
-                __syncthreads();
-                BMGD_STAMP(2);
-                T tot[FPT];
-#pragma unroll
-                for (int i = 0; i < FPT; ++i) {
-                    const int f = tid + i * nthreads;
-                    tot[i] = (f < p) ? strided_sum(gpart + f, plan.gpart_rows, PCAP) : T(0);
-                }
-                BMGD_STAMP(3);
-
-                const int parity = (int)(step_count & 1u);
-                T* cp = cpart + parity * S * PCAP;
-
-                if (cpc == 1) {
-                    // ---- one cluster per chain: push to every peer, one barrier, sum locally
-                    if (S > 1) {
-                        const uint32_t mine = smem_u32(cp + rank * PCAP);
-#pragma unroll
-                        for (int i = 0; i < FPT; ++i) {
-                            const int f = tid + i * nthreads;
-                            if (f < p)
-                                for (int peer = 0; peer < S; ++peer)
-                                    st_cluster(map_to_cta(mine + f * (uint32_t)sizeof(T), (uint32_t)peer), tot[i]);
-                        }
-                        __syncwarp();
-                        cluster_arrive_release();
-                        issue_one();  // the copies for a later stage go out while the barrier completes
-                        cluster_wait_acquire();
-#pragma unroll
-                        for (int i = 0; i < FPT; ++i) {
-                            const int f = tid + i * nthreads;
-                            tot[i] = (f < p) ? strided_sum(cp + f, S, PCAP) : T(0);
-                        }
-                    }
-                    BMGD_STAMP(4);
-                    BMGD_STAMP(5);
-#pragma unroll
-                    for (int i = 0; i < FPT; ++i) {
-                        const int f = tid + i * nthreads;
-                        if (f < p) gfin[f] = tot[i];
-                    }
-                    __syncthreads();
-                } else {
-                    // ---- several clusters per chain: reduce-scatter in the cluster, packets between the slice
-                    //      owners of different clusters, all-gather of the totals in the cluster
-                    if (S > 1) {
-                        const uint32_t mine = smem_u32(cp + rank * PCAP);
-#pragma unroll
-                        for (int i = 0; i < FPT; ++i) {
-                            const int f = tid + i * nthreads;
-                            if (f < p) st_cluster(map_to_cta(mine + f * (uint32_t)sizeof(T), (uint32_t)(f / slice)), tot[i]);
-                        }
-                        __syncwarp();
-                        cluster_arrive_release();
-                        cluster_wait_acquire();
-                    }
-                    BMGD_STAMP(4);
-                    const uint32_t tag = P.tag_base + step_count + 1u;
-                    unsigned long long* slot = P.ll + ((size_t)(team * 2 + parity) * cpc) * (size_t)P.ll_stride;
-                    // thread j of the CTA owns predictor f = rank*slice + j of the slice (all of them if S == 1)
-#pragma unroll
-                    for (int i = 0; i < FPT; ++i) {
-                        const int j = tid + i * nthreads;
-                        const int f = rank * slice + j;
-                        if (j < slice && f < p) {
-                            const T mine_sum = (S > 1) ? strided_sum(cp + f, S, PCAP) : tot[i];
-#pragma unroll
-                            for (int w = 0; w < NW; ++w)
-                                st_packet(slot + (size_t)kc * P.ll_stride + f * NW + w,
-                                          ((unsigned long long)tag << 32) | Words<T>::get(mine_sum, w));
-                        }
-                    }
-                    BMGD_STAMP(12);
-#pragma unroll
-                    for (int i = 0; i < FPT; ++i) {
-                        const int j = tid + i * nthreads;
-                        const int f = rank * slice + j;
-                        if (j >= slice || f >= p) continue;
-                        unsigned long long v[kMaxCpc][NW];
-                        unsigned long long t0 = 0;
-                        uint32_t spins = 0;
-                        while (!aborted) {
-                            // all loads first, all tag checks after: a check between two loads would make the
-                            // second load wait for the first one's round trip to L2
-#pragma unroll
-                            for (int k = 0; k < kMaxCpc; ++k) {
-                                if (k < cpc) {
-#pragma unroll
-                                    for (int w = 0; w < NW; ++w) v[k][w] = ld_packet(slot + (size_t)k * P.ll_stride + f * NW + w);
-                                }
-                            }
-                            bool ok = true;
-#pragma unroll
-                            for (int k = 0; k < kMaxCpc; ++k) {
-                                if (k < cpc) {
-#pragma unroll
-                                    for (int w = 0; w < NW; ++w) ok &= ((uint32_t)(v[k][w] >> 32) == tag);
-                                }
-                            }
-                            if (ok) break;
-                            if ((++spins & 0x3FFu) == 0u) {
-                                const unsigned long long now = global_ns();
-                                if (t0 == 0) t0 = now;
-                                if (now - t0 > P.timeout_ns || ((volatile int*)P.status)[1] != 0) {
-                                    atomicCAS(P.status, 0, kStatusTimeout);
-                                    atomicExch(P.status + 1, 1);
-                                    aborted = true;
-                                }
-                            }
-                        }
-#ifdef BMGD_TRACE
-                        if (blockIdx.x == BMGD_TRACE_BLOCK && tid == 0 && step_count < (uint32_t)kTraceSteps) {
-                            g_trace[step_count * kTracePhases + 13] = clock64();
-                            g_trace[step_count * kTracePhases + 14] = spins;
-                        }
-#endif
-                        T s = T(0);
-                        if (!aborted) {
-#pragma unroll
-                            for (int k = 0; k < kMaxCpc; ++k) {
-                                if (k < cpc) {
-                                    uint32_t w32[NW];
-#pragma unroll
-                                    for (int w = 0; w < NW; ++w) w32[w] = (uint32_t)v[k][w];
-                                    s += Words<T>::make(w32);
-                                }
-                            }
-                        }
-                        if (S > 1) {
-                            const uint32_t dst = smem_u32(gfin + f);
-                            for (int peer = 0; peer < S; ++peer) st_cluster(map_to_cta(dst, (uint32_t)peer), s);
-                        } else {
-                            gfin[f] = s;
-                        }
-                    }
-                    BMGD_STAMP(5);
-                    // The copies for a later stage go out only now: issued earlier they would sit in front of the
-                    // packet stores and polls on the same load/store path and delay the exchange by their drain time.
-                    __syncwarp();
-                    if (S > 1) {
-                        cluster_arrive_release();
-                        issue_one();
-                        cluster_wait_acquire();
-                    } else {
-                        issue_one();
-                        __syncthreads();
-                    }
-                }
-                BMGD_STAMP(6);
-
-                // ---- everyone updates its own copy of theta
-                const T scale = (min(n, N0 - sh.lo) == n) ? scale_full : scale_last;
-                {
-                    const T* gf = gfin + sub * VEC;
-#pragma unroll
-                    for (int k = 0; k < KCH; ++k) {
-                        if constexpr (CB == 16 && sizeof(T) == 4) {
-                            const float4 v = *reinterpret_cast<const float4*>(gf + k * LPR * VEC);
-                            th[k * VEC + 0] = fma(-scale, v.x, th[k * VEC + 0]);
-                            th[k * VEC + 1] = fma(-scale, v.y, th[k * VEC + 1]);
-                            th[k * VEC + 2] = fma(-scale, v.z, th[k * VEC + 2]);
-                            th[k * VEC + 3] = fma(-scale, v.w, th[k * VEC + 3]);
-                        } else {
-#pragma unroll
-                            for (int e = 0; e < VEC; ++e)
-                                th[k * VEC + e] = fma(-scale, gf[k * LPR * VEC + e], th[k * VEC + e]);
+                return (uint32_t)__popc(__ballot_sync(0xFFFFFFFFu, have));
+            } else {
+                const int iters = min(32, left + rpi - 1) / rpi;
+                for (int i = 0; i < iters; ++i) {
+                    const int sl = i * rpi + rsub;
+                    const uint32_t row = __shfl_sync(0xFFFFFFFFu, rows, sl);
+                    const bool have = row != kNoRow;
+                    const unsigned char* src = Xb + (have ? (size_t)row * row_bytes : 0);
+                    const uint32_t dst = stage_base + (uint32_t)((s0 + sl) * pitch + cl * CB);
+                    if (sl < left) {
+                        for (int k = 0; k < cpl; ++k) {
+                            const int ch = cl + k * lpr_c;
+                            if (ch < nchunks) cp_async_fill<CB>(dst + (uint32_t)(k * lpr_c * CB), src + (have ? (size_t)k * lpr_c * CB : 0), have);
                         }
                     }
                 }
-                BMGD_STAMP(7);
-                ++step_count;
+                if (lane < left) {
+                    const bool have = rows != kNoRow;
+                    cp_async_fill<(int)sizeof(T)>(stage_base + (uint32_t)((s0 + lane) * pitch + YOFF), yb + (have ? rows : 0u), have);
+                }
+                return 0u;
+            }
+        };
+        // closes this warp's part of a stage: every lane arrives once its element copies have landed, one lane
+        // announces the bytes of the warp's bulk copies
+        auto finish_stage = [&](uint32_t full_bar, uint32_t bulk_rows) {
+            mbar_arrive_after_copies(full_bar);
+            if constexpr (CB == 16) {
+                __syncwarp();  // the zero fills of all lanes come before the announcing lane's arrival
+                if (lane == 0) mbar_arrive_expect_tx(full_bar, bulk_rows * row_bytes);
+            }
+        };
+
+        uint32_t rot = (uint32_t)pw;  // (pw - pair * nbatch) mod NPW, kept incrementally: ownership of batches rotates
+        const uint32_t rot_step = (uint32_t)(nbatch % NPW);
+        for (uint32_t it = 0; it < total_stages; it += 2) {
+            const Cursor A = cur;
+            advance(cur);
+            const bool two = it + 1 < total_stages;
+            const Cursor B = cur;
+            if (two) advance(cur);
+            const int slotA = slot;
+            const uint32_t parA = empty_parity;
+            if (++slot == D) { slot = 0; empty_parity ^= 1u; }
+            const int slotB = slot;
+            const uint32_t parB = empty_parity;
+            if (two && ++slot == D) { slot = 0; empty_parity ^= 1u; }
+            const uint32_t baseA = ring_base + (uint32_t)(slotA * stage_bytes), baseB = ring_base + (uint32_t)(slotB * stage_bytes);
+            const int b0 = (int)rot;  // this producer's first batch in this pair of stages
+            rot = (rot + (uint32_t)NPW - rot_step) % (uint32_t)NPW;
+
+            // the shuffle of both stages first (it needs no ring slot), then the copies of A, then those of B
+            uint32_t rowsA[kMaxBatchesPerProducer], rowsB[kMaxBatchesPerProducer];
+#pragma unroll
+            for (int kk = 0; kk < kMaxBatchesPerProducer; ++kk) {
+                const int bb = b0 + kk * NPW;
+                rowsA[kk] = kNoRow; rowsB[kk] = kNoRow;
+                if (bb < nbatch) {
+                    const int s = 32 * bb + lane;
+                    const uint32_t ua = (uint32_t)(A.sidx * R + s), ub = (uint32_t)(B.sidx * R + s);
+                    const bool va = s < R && ua < A.sh.cnt;
+                    const bool vb = two && s < R && ub < B.sh.cnt;
+                    uint32_t ra = va ? A.sh.lo + A.sh.a + ua : 0u, rb_ = vb ? B.sh.lo + B.sh.a + ub : 0u;
+                    if (__any_sync(0xFFFFFFFFu, va || vb)) perm_index2(ra, A.rk, rb_, B.rk, dom);
+                    __syncwarp();  // lanes walked the cycle for different lengths
+                    if (va) rowsA[kk] = ra;
+                    if (vb) rowsB[kk] = rb_;
+                }
+            }
+            const uint32_t fullA = full_bars + (uint32_t)(slotA * 8), fullB = full_bars + (uint32_t)(slotB * 8);
+            bounded_mbar_wait(empty_bars + (uint32_t)(slotA * 8), parA, aborted, P);
+            __syncwarp();
+            uint32_t sent = 0;
+#pragma unroll
+            for (int kk = 0; kk < kMaxBatchesPerProducer; ++kk) {
+                const int bb = b0 + kk * NPW;
+                if (bb < nbatch) sent += copy_batch(baseA, fullA, 32 * bb, rowsA[kk]);
+            }
+            finish_stage(fullA, sent);  // a producer without a batch in this stage still counts on its barrier
+            if (two) {
+                bounded_mbar_wait(empty_bars + (uint32_t)(slotB * 8), parB, aborted, P);
+                __syncwarp();
+                sent = 0;
+#pragma unroll
+                for (int kk = 0; kk < kMaxBatchesPerProducer; ++kk) {
+                    const int bb = b0 + kk * NPW;
+                    if (bb < nbatch) sent += copy_batch(baseB, fullB, 32 * bb, rowsB[kk]);
+                }
+                finish_stage(fullB, sent);
             }
         }
+        cp_async_wait_all();
+    } else {
+        // ================================================================ consumer warps
+        const int grp = lane / LPR, sub = lane % LPR;
+        const int nchunks = p / VEC;
+        T* gpart = reinterpret_cast<T*>(smem + plan.gpart_off);
+        T* gfin = reinterpret_cast<T*>(smem + plan.gfin_off);
+        const uint32_t cpk_base = smem_u32(smem + plan.cpk_off), gpk_base = smem_u32(smem + plan.gpk_off);
+        const int lane_off = (warp * GPW + grp) * pitch + sub * CB;  // this lane's first chunk inside a sub-pass
+        const int subpass_bytes = spp * pitch;
+        const int y_rel = YOFF - sub * CB;
+        const uint32_t warp_first = (uint32_t)(warp * GPW);  // first row slot of this warp in sub-pass 0
+        const int slice = (p + S - 1) / S;  // predictors owned by one CTA of a cluster in the sliced exchange
+        const T scale_full = (T)P.scale_full, scale_last = (T)P.scale_last;
 
-        if (g == 0 && warp == 0 && grp == 0) {
+        int cs_slot = 0;         // ring slot the compute cursor reads next
+        uint32_t cs_phase = 0;   // parity of that slot's "full" phase
+        uint32_t step_count = 0; // steps this team has finished in this launch
+
+        for (int ci = 0; ci < nch; ++ci) {
+            const int chain = team + ci * P.nteams;
+            T* theta_g = static_cast<T*>(P.theta) + (size_t)chain * p;
+
+            T th[NV];
 #pragma unroll
             for (int k = 0; k < KCH; ++k) {
                 const int c = sub + k * LPR;
-                if (c < nchunks)
 #pragma unroll
-                    for (int e = 0; e < VEC; ++e) theta_g[c * VEC + e] = th[k * VEC + e];
+                for (int e = 0; e < VEC; ++e) th[k * VEC + e] = (c < nchunks) ? theta_g[c * VEC + e] : T(0);
+            }
+
+            for (int t = 0; t < T_rounds; ++t) {
+                for (uint32_t m = 0; m < M; ++m) {
+                    const RowShare sh = row_share(m, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full);
+                    BMGD_STAMP(0);
+
+                    T gacc[NV];
+#pragma unroll
+                    for (int i = 0; i < NV; ++i) gacc[i] = T(0);
+
+                    // sub-passes of this step in which the warp has at least one row
+                    int sp_left = (sh.cnt > warp_first) ? (int)((sh.cnt - warp_first - 1u) / (uint32_t)spp) + 1 : 0;
+                    for (int sidx = 0; sidx < passes; ++sidx) {
+                        bounded_mbar_wait(full_bars + (uint32_t)(cs_slot * 8), cs_phase, aborted, P);
+                        __syncwarp();
+                        const unsigned char* rowp = smem + plan.ring_off + cs_slot * stage_bytes + lane_off;
+                        int nsub = min(sp_left, RB);
+                        sp_left -= nsub;
+                        if constexpr (NV * (int)sizeof(T) <= 32) {  // narrow rows: four independent rows in flight per group
+                            for (; nsub >= 4; nsub -= 4, rowp += 4 * subpass_bytes) {
+                                row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, y_rel, th, gacc);
+                                row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + subpass_bytes, y_rel, th, gacc);
+                                row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + 2 * subpass_bytes, y_rel, th, gacc);
+                                row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + 3 * subpass_bytes, y_rel, th, gacc);
+                            }
+                        }
+                        for (; nsub >= 2; nsub -= 2, rowp += 2 * subpass_bytes) {  // two independent rows in flight per group
+                            row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, y_rel, th, gacc);
+                            row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + subpass_bytes, y_rel, th, gacc);
+                        }
+                        if (nsub) row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, y_rel, th, gacc);
+                        __syncwarp();  // every lane has its values in registers: the slot may be refilled
+                        if (lane == 0) mbar_arrive(empty_bars + (uint32_t)(cs_slot * 8));
+                        if (++cs_slot == D) { cs_slot = 0; cs_phase ^= 1u; }
+                    }
+                    BMGD_STAMP(1);
+
+                    // ---- sum the partial gradients of this CTA in fixed order
+                    if constexpr (PRE) {
+#pragma unroll
+                        for (int off = LPR; off < 32; off <<= 1)
+#pragma unroll
+                            for (int i = 0; i < NV; ++i) gacc[i] += __shfl_xor_sync(0xFFFFFFFFu, gacc[i], off);
+                    }
+                    if (!PRE || grp == 0) {
+                        T* gp = gpart + (PRE ? warp : warp * GPW + grp) * PCAP + sub * VEC;
+#pragma unroll
+                        for (int k = 0; k < KCH; ++k) {
+                            if constexpr (CB == 16 && sizeof(T) == 4)
+                                *reinterpret_cast<float4*>(gp + k * LPR * VEC) =
+                                    make_float4(gacc[k * VEC], gacc[k * VEC + 1], gacc[k * VEC + 2], gacc[k * VEC + 3]);
+                            else if constexpr (CB == 16)
+                                *reinterpret_cast<double2*>(gp + k * LPR * VEC) = make_double2(gacc[k * VEC], gacc[k * VEC + 1]);
+                            else
+                                gp[k * LPR] = gacc[k];
+                        }
+                    }
+                    consumer_sync(nthreads);
+                    BMGD_STAMP(2);
+                    T tot[FPT];
+#pragma unroll
+                    for (int i = 0; i < FPT; ++i) {
+                        const int f = tid + i * nthreads;
+                        tot[i] = (f < p) ? strided_sum(gpart + f, plan.gpart_rows, PCAP) : T(0);
+                    }
+                    BMGD_STAMP(3);
+
+                    const int parity = (int)(step_count & 1u);
+                    // Tag of this step's packets, in shared memory (zeroed at launch) and in global memory (tags of
+                    // earlier launches are smaller): never 0, never repeated while a packet of the same slot can be read.
+                    const uint32_t tag = P.tag_base + step_count + 1u;
+                    const uint32_t cpk = cpk_base + (uint32_t)(parity * S * plan.cpk_stride * 8);
+
+                    if (cpc == 1) {
+                        // ---- one cluster per chain: every CTA pushes its partial sums, as tagged packets, into the
+                        //      shared memory of every CTA of the cluster and then sums, in rank order, the S packets per
+                        //      predictor that arrive in its own.  No cluster barrier: a packet is its own flag.
+                        if (S > 1) {
+    #pragma unroll
+                            for (int i = 0; i < FPT; ++i) {
+                                const int f = tid + i * nthreads;
+                                if (f < p) {
+    #pragma unroll
+                                    for (int w = 0; w < NW; ++w) {
+                                        const unsigned long long pk = ((unsigned long long)tag << 32) | Words<T>::get(tot[i], w);
+                                        const uint32_t mine = cpk + (uint32_t)((rank * plan.cpk_stride + f * NW + w) * 8);
+                                        for (int peer = 0; peer < S; ++peer) st_cluster_u64(map_to_cta(mine, (uint32_t)peer), pk);
+                                    }
+                                }
+                            }
+    #pragma unroll
+                            for (int i = 0; i < FPT; ++i) {
+                                const int f = tid + i * nthreads;
+                                if (f < p)
+                                    tot[i] = gather_packets<T, kMaxClusterSize, 4>(
+                                        S, tag, aborted, P,
+                                        [&](int k, int w) { return ld_shared_volatile_u64(cpk + (uint32_t)((k * plan.cpk_stride + f * NW + w) * 8)); });
+                            }
+                        }
+                        BMGD_STAMP(4);
+                        BMGD_STAMP(5);
+    #pragma unroll
+                        for (int i = 0; i < FPT; ++i) {
+                            const int f = tid + i * nthreads;
+                            if (f < p) gfin[f] = tot[i];
+                        }
+                        consumer_sync(nthreads);
+                    } else {
+                        // ---- several clusters per chain: reduce-scatter in the cluster (CTA r owns a slice of the
+                        //      predictors and receives its peers' partial sums as tagged packets), packets through global
+                        //      memory between the slice owners of different clusters, totals pushed to every peer
+                        if (S > 1) {
+    #pragma unroll
+                            for (int i = 0; i < FPT; ++i) {
+                                const int f = tid + i * nthreads;
+                                if (f < p) {
+                                    const int owner = f / slice;
+    #pragma unroll
+                                    for (int w = 0; w < NW; ++w)
+                                        st_cluster_u64(map_to_cta(cpk + (uint32_t)((rank * plan.cpk_stride + (f - owner * slice) * NW + w) * 8),
+                                                                  (uint32_t)owner),
+                                                       ((unsigned long long)tag << 32) | Words<T>::get(tot[i], w));
+                                }
+                            }
+                        }
+                        BMGD_STAMP(4);
+                        unsigned long long* slot = P.ll + ((size_t)(team * 2 + parity) * cpc) * (size_t)P.ll_stride;
+                        const uint32_t gpk = gpk_base + (uint32_t)(parity * PCAP * NW * 8);
+                        // thread j of the CTA owns predictor f = rank*slice + j of the slice (all of them if S == 1)
+    #pragma unroll
+                        for (int i = 0; i < FPT; ++i) {
+                            const int j = tid + i * nthreads;
+                            const int f = rank * slice + j;
+                            if (j < slice && f < p) {
+                                const T mine_sum = (S > 1)
+                                    ? gather_packets<T, kMaxClusterSize, 4>(
+                                          S, tag, aborted, P,
+                                          [&](int k, int w) { return ld_shared_volatile_u64(cpk + (uint32_t)((k * plan.cpk_stride + j * NW + w) * 8)); })
+                                    : tot[i];
+    #pragma unroll
+                                for (int w = 0; w < NW; ++w)
+                                    st_packet(slot + (size_t)kc * P.ll_stride + f * NW + w,
+                                              ((unsigned long long)tag << 32) | Words<T>::get(mine_sum, w));
+                            }
+                        }
+                        BMGD_STAMP(12);
+    #pragma unroll
+                        for (int i = 0; i < FPT; ++i) {
+                            const int j = tid + i * nthreads;
+                            const int f = rank * slice + j;
+                            if (j >= slice || f >= p) continue;
+                            const unsigned long long* src = slot + f * NW;
+                            const int stride = P.ll_stride;
+                            const T s = gather_packets<T, kMaxCpc, kMaxCpc>(
+                                cpc, tag, aborted, P, [&](int k, int w) { return ld_packet(src + (size_t)k * stride + w); });
+                            if (S > 1) {
+    #pragma unroll
+                                for (int w = 0; w < NW; ++w) {
+                                    const unsigned long long pk = ((unsigned long long)tag << 32) | Words<T>::get(s, w);
+                                    const uint32_t dst = gpk + (uint32_t)((f * NW + w) * 8);
+                                    for (int peer = 0; peer < S; ++peer) st_cluster_u64(map_to_cta(dst, (uint32_t)peer), pk);
+                                }
+                            } else {
+                                gfin[f] = s;
+                            }
+                        }
+                        BMGD_STAMP(5);
+                        if (S > 1) {
+    #pragma unroll
+                            for (int i = 0; i < FPT; ++i) {
+                                const int f = tid + i * nthreads;
+                                if (f < p)
+                                    gfin[f] = gather_packets<T, 1, 1>(
+                                        1, tag, aborted, P,
+                                        [&](int, int w) { return ld_shared_volatile_u64(gpk + (uint32_t)((f * NW + w) * 8)); });
+                            }
+                        }
+                        consumer_sync(nthreads);
+                    }
+                    BMGD_STAMP(6);
+
+                    // ---- everyone updates its own copy of theta
+                    const T scale = (min(n, N0 - sh.lo) == n) ? scale_full : scale_last;
+                    {
+                        const T* gf = gfin + sub * VEC;
+#pragma unroll
+                        for (int k = 0; k < KCH; ++k) {
+                            if constexpr (CB == 16 && sizeof(T) == 4) {
+                                const float4 v = *reinterpret_cast<const float4*>(gf + k * LPR * VEC);
+                                th[k * VEC + 0] = fma(-scale, v.x, th[k * VEC + 0]);
+                                th[k * VEC + 1] = fma(-scale, v.y, th[k * VEC + 1]);
+                                th[k * VEC + 2] = fma(-scale, v.z, th[k * VEC + 2]);
+                                th[k * VEC + 3] = fma(-scale, v.w, th[k * VEC + 3]);
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < VEC; ++e)
+                                    th[k * VEC + e] = fma(-scale, gf[k * LPR * VEC + e], th[k * VEC + e]);
+                            }
+                        }
+                    }
+                    BMGD_STAMP(7);
+                    ++step_count;
+                }
+            }
+
+            if (g == 0 && warp == 0 && grp == 0) {
+#pragma unroll
+                for (int k = 0; k < KCH; ++k) {
+                    const int c = sub + k * LPR;
+                    if (c < nchunks)
+#pragma unroll
+                        for (int e = 0; e < VEC; ++e) theta_g[c * VEC + e] = th[k * VEC + e];
+                }
             }
         }
     }
-    cp_async_wait_all();
+    if (S > 1) {  // no CTA leaves while a peer's packets for it may still be on their way
+        __syncwarp();
+        cluster_arrive_release();
+        cluster_wait_acquire();
+    }
 }
 
 // Waits, with the step kernel's protocol, for a packet tag that nobody writes: the wait must run out of its

@@ -81,28 +81,28 @@ def test_launch_shapes_agree_with_the_oracle(shape):
 
 
 @pytest.mark.parametrize("shape", [
-    dict(cluster_size=1, ctas_per_chain=1),
-    dict(cluster_size=2, ctas_per_chain=12),
-    dict(cluster_size=8, ctas_per_chain=8, threads_per_cta=512),
-    dict(cluster_size=8, ctas_per_chain=16, pipeline_depth=2, subpasses_per_stage=4),
-    dict(cluster_size=16, ctas_per_chain=32),
+    dict(cluster_size=1, ctas_per_chain=1, producer_warps=1),
+    dict(cluster_size=2, ctas_per_chain=12, producer_warps=2),
+    dict(cluster_size=8, ctas_per_chain=8, threads_per_cta=512, producer_warps=3),
+    dict(cluster_size=8, ctas_per_chain=8, threads_per_cta=512, producer_warps=1),
+    dict(cluster_size=8, ctas_per_chain=16, pipeline_depth=2, subpasses_per_stage=4, producer_warps=2),
+    dict(cluster_size=4, ctas_per_chain=4, pipeline_depth=8, subpasses_per_stage=1, producer_warps=1),
+    dict(cluster_size=16, ctas_per_chain=32, producer_warps=2),
 ])
-def test_bulk_copy_rows_agree_with_the_oracle(shape):
-    """The same launches with every row fetched by one cp.async.bulk onto a per-warp mbarrier."""
-    from paper_2312_08728_b200.binding import FLAG_BULK_ROWS
-    check(SMALL, buffers_of(SMALL), mode="resident", flags=FLAG_BULK_ROWS, **shape)
+def test_producer_warp_counts_and_ring_depths_agree_with_the_oracle(shape):
+    """Rows are fetched by dedicated warps: any number of them, and any ring depth, must give the same theta."""
+    check(SMALL, buffers_of(SMALL), mode="resident", **shape)
     w = WORKLOADS["cfg1"].scaled(N=4_000, K=2, epochs=1)
-    check(w, buffers_of(w), mode="slots", flags=FLAG_BULK_ROWS)
+    check(w, buffers_of(w), mode="slots", producer_warps=shape["producer_warps"])
 
 
-def test_bulk_copy_rows_ragged_and_chains():
-    from paper_2312_08728_b200.binding import FLAG_BULK_ROWS
+def test_producer_warps_ragged_batches_and_chains():
     w = WORKLOADS["cfg3"].scaled(N=100_000, K=2, T=2, epochs=1)
-    check(w, buffers_of(w), flags=FLAG_BULK_ROWS)
+    check(w, buffers_of(w), producer_warps=1)
     w = WORKLOADS["cfg2"].scaled(N=60_000, K=3, T=2, epochs=1, Rc=8)
-    check(w, buffers_of(w), mode="resident", flags=FLAG_BULK_ROWS)
+    check(w, buffers_of(w), mode="resident", producer_warps=3)
     w = Workload("edge", LOSS_LINEAR, DTYPE_F64, N=257, p=6, K=1, n=3, T=2, lr=0.1, epochs=1, rho=0.5, seed=9)
-    check(w, buffers_of(w), mode="resident", flags=FLAG_BULK_ROWS)
+    check(w, buffers_of(w), mode="resident", producer_warps=1)
 
 
 def test_cluster_of_sixteen_if_the_device_allows_it():
