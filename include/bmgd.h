@@ -88,7 +88,7 @@ typedef struct bmgd_config {
     int32_t threads_per_cta;  /* threads that compute: a multiple of 32 from 256 to 512 (softmax: 256, 512 or 1024) */
     int32_t pipeline_depth;   /* row-prefetch stages held in shared memory: 2 to 8 */
     int32_t subpasses_per_stage; /* a stage holds this many sweeps of the CTA over its rows: 1, 2, 4, ... 32 */
-    int32_t producer_warps;   /* linear/logistic: extra warps per CTA that only evaluate the shuffle and fetch rows: 1 to 4 */
+    int32_t producer_warps;   /* linear/logistic: extra warps per CTA that only evaluate the shuffle and fetch rows: 1 to 8 */
     int32_t reserved[6];      /* must be zero */
 } bmgd_config;
 

@@ -112,7 +112,7 @@ int validate(const bmgd_config* c) {
     if (N0 > 0x7FFFFFFFll) return BMGD_ERR_ARG;
     for (int i = 0; i < 6; ++i)
         if (c->reserved[i] != 0) return BMGD_ERR_ARG;
-    if (c->producer_warps < 0 || c->producer_warps > 4) return BMGD_ERR_ARG;
+    if (c->producer_warps < 0 || c->producer_warps > 8) return BMGD_ERR_ARG;
     if (c->cluster_size != 0 && c->cluster_size != 1 && c->cluster_size != 2 && c->cluster_size != 4 &&
         c->cluster_size != 8 && c->cluster_size != 16)
         return BMGD_ERR_ARG;
@@ -149,9 +149,47 @@ Layout make_layout(const bmgd_config* c) {
     return L;
 }
 
+// ------------------------------------------------------------------ tensor map of a buffer
+
+// cuTensorMapEncodeTiled, looked up through the runtime so that the library links against cudart only.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static std::once_flag once;
+    static EncodeTiledFn fn = nullptr;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            cudaGetLastError();
+    });
+    return fn;
+}
+
+// X [rows][p] as a 2-D tensor whose box is one row of `box` values (the kernel's predictor capacity): the step kernel
+// gathers four rows per copy; columns from p on, and rows from `rows` on, read as zeros.  dev_x and the row size are
+// 16-byte multiples.  Host-only work: nothing is allocated.
+int make_row_map(const void* dev_x, int64_t rows, int p, int elem_bytes, int box, CUtensorMap* out) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return BMGD_ERR_CUDA;
+    const cuuint64_t dims[2] = {(cuuint64_t)p, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)p * (cuuint64_t)elem_bytes};
+    const cuuint32_t boxdim[2] = {(cuuint32_t)box, 1u};
+    const cuuint32_t estr[2] = {1u, 1u};
+    const CUresult r = enc(out, elem_bytes == 8 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT64 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                           const_cast<void*>(dev_x), dims, strides, boxdim, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? BMGD_OK : BMGD_ERR_CUDA;
+}
+
 // ------------------------------------------------------------------ GLM kernel table
 
-typedef void (*GlmKernel)(const GlmParams);
+typedef void (*GlmKernel)(const GlmParams, const CUtensorMap);
 
 struct GlmVariant {
     GlmKernel fn;
@@ -217,8 +255,11 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     const int gpw = 32 / var->lpr;
     const int pcap = var->cap();
     LaunchShape L{};
-    L.threads = c.threads_per_cta ? std::min(c.threads_per_cta, var->max_consumer_threads())
-                                  : ((c.Rc > 1 && var->max_consumer_threads() >= 512) ? 512 : 256);
+    // Replicate chains keep every SM busy with several chains' rows in flight: throughput, not the per-step latency,
+    // sets the pace there, so the CTA is as large as the register file allows (measured on B200: 16 consumer warps
+    // and 4 producer warps beat 12 + 8 and 14 + 6 once rows arrive four per gather).
+    const bool throughput = c.Rc > 1 && var->max_consumer_threads() >= 512;
+    L.threads = c.threads_per_cta ? std::min(c.threads_per_cta, var->max_consumer_threads()) : (throughput ? 512 : 256);
     // Producer warps only evaluate the shuffle and issue copies; both are chains of dependent instructions, so several
     // warps side by side are what keeps them ahead of the consumers.
     L.pwarps = c.producer_warps ? c.producer_warps : 4;
@@ -227,7 +268,7 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     const int warps = L.threads / 32;
     const int spp = warps * gpw;  // rows a CTA works on at once (one sub-pass)
     const bool pre = var->kch * var->vec <= 16;
-    const int pitch = pcap * eb + 16;
+    const bool gathered = bmgdk::glm_gathered(var->vec * eb, pcap);
 
     // Cluster size.  Measured on B200: a step costs one cluster barrier (about 0.6-0.9 us) inside one cluster, and
     // about 2.5 us more once partial sums have to cross clusters through L2, while a sub-pass of spp rows costs about
@@ -245,9 +286,9 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     // the largest ring we would use (a smaller one can only admit more).
     int max_clusters = 0, fixed_smem = 0, ring_budget = 0;
     for (;;) {
-        fixed_smem = bmgdk::glm_smem_plan(warps, gpw, pre, 1, 0, pcap, eb, S, false).total_bytes;
+        fixed_smem = bmgdk::glm_smem_plan(warps, gpw, pre, 1, 0, pcap, eb, S, false, gathered).total_bytes;
         ring_budget = std::min(h->smem_optin - fixed_smem, 160 * 1024);
-        if (ring_budget < 2 * spp * pitch) {  // the per-peer exchange buffers of a large cluster leave no room for rows
+        if (ring_budget < 2 * bmgdk::glm_smem_plan(warps, gpw, pre, 1, 1, pcap, eb, S, false, gathered).stage_bytes) {  // the per-peer exchange buffers of a large cluster leave no room for rows
             if (c.cluster_size == 0 && S > 1) { S /= 2; continue; }
             return BMGD_ERR_UNIMPLEMENTED;
         }
@@ -288,7 +329,7 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     }
     // a chain that spans clusters keeps only its slice of the peers' packets in shared memory: more room for rows
     const bool multi = L.cpc > 1;
-    fixed_smem = bmgdk::glm_smem_plan(warps, gpw, pre, 1, 0, pcap, eb, S, multi).total_bytes;
+    fixed_smem = bmgdk::glm_smem_plan(warps, gpw, pre, 1, 0, pcap, eb, S, multi, gathered).total_bytes;
     ring_budget = std::min(h->smem_optin - fixed_smem, 160 * 1024);
     const int G = L.cpc * S;
     const int rows_per_cta = (n + G - 1) / G;
@@ -296,22 +337,22 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
 
     // sub-passes per ring stage: two or more let a group keep two rows in flight and amortise the per-stage
     // bookkeeping; measured on B200, two stages of two sub-passes beat four stages of one when rows come from L2
-    const int subpass_bytes = spp * pitch;
+    auto stage_bytes_of = [&](int r) { return bmgdk::glm_smem_plan(warps, gpw, pre, r, 1, pcap, eb, S, multi, gathered).stage_bytes; };
     // narrow rows (at most 32 bytes per lane) are swept four sub-passes at a time by the kernel, others two
     int rb = c.subpasses_per_stage ? c.subpasses_per_stage : ((var->kch * 16 <= 32) ? 4 : 2);
     rb = floor_pow2(std::max(1, std::min(rb, subpasses)));
     // a producer warp takes at most kMaxBatchesPerProducer batches of 32 row slots per stage
     while (rb > 1 && rb * spp > 32 * bmgdk::kMaxBatchesPerProducer * L.pwarps) rb /= 2;
     if (spp > 32 * bmgdk::kMaxBatchesPerProducer * L.pwarps) return BMGD_ERR_ARG;
-    while (rb > 1 && 2 * rb * subpass_bytes > ring_budget) rb /= 2;
+    while (rb > 1 && 2 * stage_bytes_of(rb) > ring_budget) rb /= 2;
     L.rb = rb;
     L.passes = (subpasses + rb - 1) / rb;
-    const int stage_bytes = rb * subpass_bytes;
+    const int stage_bytes = stage_bytes_of(rb);
     int depth = c.pipeline_depth ? c.pipeline_depth : 4;  // ring stages: 2 to 8
     while (depth > 2 && depth * stage_bytes > ring_budget) --depth;
     if (depth * stage_bytes > ring_budget) return BMGD_ERR_UNIMPLEMENTED;
     L.depth = depth;
-    L.smem = bmgdk::glm_smem_plan(warps, gpw, pre, rb, depth, pcap, eb, S, multi).total_bytes;
+    L.smem = bmgdk::glm_smem_plan(warps, gpw, pre, rb, depth, pcap, eb, S, multi, gathered).total_bytes;
     (void)rows;
     *out = L;
     return BMGD_OK;
@@ -416,7 +457,16 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
         if (rc != BMGD_OK) return rc;
         BMGD_CUDA(h, cudaEventRecord(ep.a, h->compute));
     }
-    cudaError_t e = cudaLaunchKernelEx(&lc, var->fn, P);
+    CUtensorMap xmap;
+    std::memset(&xmap, 0, sizeof xmap);
+    if (bmgdk::glm_gathered(var->vec * h->tb, var->cap())) {
+        rc = make_row_map(dx, rows, c.p, h->tb, var->cap(), &xmap);
+        if (rc != BMGD_OK) {
+            if (timing) h->event_pool.push_back(ep);
+            return rc;
+        }
+    }
+    cudaError_t e = cudaLaunchKernelEx(&lc, var->fn, P, xmap);
     if (e != cudaSuccess) {
         h->last_cuda = (int)e;
         cudaGetLastError();
@@ -838,7 +888,13 @@ int bmgd_run_rounds_noalloc(const void* dev_x, const void* dev_y, int64_t rows, 
         ++na;
     }
     lc.attrs = at; lc.numAttrs = (unsigned)na;
-    cudaError_t e = cudaLaunchKernelEx(&lc, var->fn, P);
+    CUtensorMap xmap;  // encoded on the host, passed by value: no allocation
+    std::memset(&xmap, 0, sizeof xmap);
+    if (bmgdk::glm_gathered(var->vec * tb, var->cap())) {
+        rc = make_row_map(dev_x, rows, p, tb, var->cap(), &xmap);
+        if (rc != BMGD_OK) return rc;
+    }
+    cudaError_t e = cudaLaunchKernelEx(&lc, var->fn, P, xmap);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return (e == cudaErrorCooperativeLaunchTooLarge || e == cudaErrorLaunchOutOfResources) ? BMGD_ERR_LAUNCH : BMGD_ERR_CUDA;

@@ -26,6 +26,7 @@
 // BMGD_ERR_TIMEOUT in the status word, stops waiting for the rest of the launch and returns.
 #pragma once
 #include <cstdint>
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include "shuffle.cuh"
@@ -139,6 +140,14 @@ __device__ __forceinline__ void bulk_copy_row(uint32_t dst_smem, const void* src
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
+// four rows of a 2-D tensor map (box: one row of `box` values), rows y0..y3 from column x on, land back to back at
+// dst (128-byte aligned); rows or columns outside the tensor read as zero; 4 * box bytes are counted on `bar`
+__device__ __forceinline__ void tma_gather4_rows(uint32_t dst_smem, const void* tmap, int x, int y0, int y1, int y2, int y3,
+                                                 uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
+                 " [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+                 ::"r"(dst_smem), "l"(tmap), "r"(x), "r"(y0), "r"(y1), "r"(y2), "r"(y3), "r"(bar) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -198,8 +207,9 @@ template <> struct Words<double> {
 // ---------------------------------------------------------------- shared-memory plan (host and device agree on it)
 
 struct GlmSmemPlan {
-    int pitch;             // bytes from one ring row to the next: the full predictor capacity, then 16 bytes for y
-    int warp_stage_bytes;  // one warp's share of one ring stage
+    int pitch;             // bytes from one ring row to the next
+    int stage_bytes;       // one ring stage: rb sub-passes of warps*gpw rows (and, in the gathered layout, their y values)
+    int stage_y_off;       // gathered layout: where the y values of a stage start inside it
     int ring_off, ring_bytes;
     int gpart_rows;        // partial-gradient rows summed per CTA
     int gpart_off, gfin_off;
@@ -208,15 +218,22 @@ struct GlmSmemPlan {
     int total_bytes;
 };
 
+// Rows of at most 256 values that are 16-byte multiples are fetched four at a time by the tensor-map gather; its
+// four rows land back to back, so a ring row is exactly the predictor capacity wide and y lives in a per-stage array.
+// Otherwise a ring row is the predictor capacity plus 16 bytes that hold y.
+__host__ __device__ constexpr bool glm_gathered(int chunk_bytes, int pcap) { return chunk_bytes == 16 && pcap <= 256; }
+
 // `multi`: a chain spans several clusters, so a CTA receives only its slice of the predictors from its peers.
 __host__ __device__ inline GlmSmemPlan glm_smem_plan(int warps, int gpw, bool prereduce, int rb, int depth, int pcap,
-                                                     int elem_bytes, int S, bool multi) {
+                                                     int elem_bytes, int S, bool multi, bool gathered) {
     GlmSmemPlan s;
     const int words = elem_bytes / 4;
-    s.pitch = pcap * elem_bytes + 16;
-    s.warp_stage_bytes = rb * gpw * s.pitch;
-    s.ring_off = 1024;  // room for one mbarrier per (warp, stage) in front of the ring
-    s.ring_bytes = warps * depth * s.warp_stage_bytes;
+    const int R = rb * warps * gpw;
+    s.pitch = gathered ? pcap * elem_bytes : pcap * elem_bytes + 16;
+    s.stage_y_off = R * s.pitch;
+    s.stage_bytes = gathered ? s.stage_y_off + (R * elem_bytes + 127) / 128 * 128 : s.stage_y_off;
+    s.ring_off = 1024;  // the stages' mbarriers sit in front of the ring
+    s.ring_bytes = depth * s.stage_bytes;
     s.gpart_rows = prereduce ? warps : warps * gpw;
     s.gpart_off = s.ring_off + s.ring_bytes;
     s.gfin_off = s.gpart_off + s.gpart_rows * pcap * elem_bytes;
@@ -372,9 +389,9 @@ __device__ __forceinline__ T strided_sum(const T* col, int rows, int stride) {
 }
 
 // One row per LPR-lane group: residual from the dot product with theta, then g += r * x.
-// `rowp` is this lane's first chunk of the row in shared memory; y sits y_rel bytes from it.
+// `rowp` is this lane's first chunk of the row in shared memory, `yp` the row's y.
 template <typename T, int VEC, int LPR, int KCH, bool LOGISTIC>
-__device__ __forceinline__ void row_step(const unsigned char* rowp, int y_rel, const T (&th)[KCH * VEC],
+__device__ __forceinline__ void row_step(const unsigned char* rowp, const unsigned char* yp, const T (&th)[KCH * VEC],
                                          T (&gacc)[KCH * VEC]) {
     constexpr int NV = KCH * VEC;
     constexpr int CB = VEC * (int)sizeof(T);
@@ -391,7 +408,7 @@ __device__ __forceinline__ void row_step(const unsigned char* rowp, int y_rel, c
             x[k] = *reinterpret_cast<const T*>(rowp + k * LPR * CB);
         }
     }
-    const T yv = *reinterpret_cast<const T*>(rowp + y_rel);
+    const T yv = *reinterpret_cast<const T*>(yp);
     T part[VEC];
 #pragma unroll
     for (int e = 0; e < VEC; ++e) part[e] = T(0);
@@ -441,7 +458,8 @@ __device__ __forceinline__ void bounded_mbar_wait(uint32_t bar, uint32_t parity,
 // inner loop carries no predicates.  Each stage has a "full" mbarrier (the producers' copies have landed) and an
 // "empty" one (every consumer warp has read it).
 template <typename T, int VEC, int LPR, int KCH, bool LOGISTIC>
-__global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(const GlmParams P) {
+__global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1)
+glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
     constexpr int GPW = 32 / LPR;            // row groups per warp
     constexpr int NV = KCH * VEC;            // values per lane
     constexpr int PCAP = LPR * KCH * VEC;    // predictor capacity
@@ -449,10 +467,11 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
     constexpr int CB = VEC * (int)sizeof(T); // copy chunk bytes
     constexpr int NW = Words<T>::N;
     constexpr bool PRE = glm_prereduce<VEC, KCH>();
-    constexpr int YOFF = PCAP * (int)sizeof(T);  // y sits behind the predictors of its row
+    constexpr bool G4 = glm_gathered(CB, PCAP);  // rows arrive four at a time through the tensor map `xmap` of X
+    constexpr int YOFF = PCAP * (int)sizeof(T);  // other layouts: y sits behind the predictors of its row
     constexpr uint32_t kNoRow = 0xFFFFFFFFu;
 
-    extern __shared__ __align__(16) unsigned char smem[];
+    extern __shared__ __align__(1024) unsigned char smem[];  // gathers want 128-byte aligned destinations
 
     const int tid = threadIdx.x;
     const int W = P.consumer_warps, NPW = P.producer_warps;  // blockDim.x == 32 * (W + NPW)
@@ -468,9 +487,9 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
     const int T_rounds = P.T, passes = P.passes, RB = P.rb, D = P.depth;
     const int spp = W * GPW;  // rows the CTA works on at once (one sub-pass)
 
-    const GlmSmemPlan plan = glm_smem_plan(W, GPW, PRE, RB, D, PCAP, (int)sizeof(T), S, cpc > 1);
+    const GlmSmemPlan plan = glm_smem_plan(W, GPW, PRE, RB, D, PCAP, (int)sizeof(T), S, cpc > 1, G4);
     const int pitch = plan.pitch;
-    const int stage_bytes = W * plan.warp_stage_bytes;
+    const int stage_bytes = plan.stage_bytes;
     const uint32_t full_bars = smem_u32(smem), empty_bars = smem_u32(smem) + 128u;  // one 8-byte mbarrier per stage each
     const int nch = (team < P.Rc) ? (P.Rc - team + P.nteams - 1) / P.nteams : 0;
     const uint32_t total_stages = (uint32_t)nch * (uint32_t)T_rounds * M * (uint32_t)passes;  // the host keeps this below 2^32
@@ -546,7 +565,23 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
         // return value is the number of rows this warp sent that way); others go element by element.
         auto copy_batch = [&](uint32_t stage_base, uint32_t full_bar, int s0, uint32_t rows) -> uint32_t {
             const int left = R - s0;  // slots of this batch that exist
-            if constexpr (CB == 16) {
+            if constexpr (G4) {
+                // lane l < 8 fetches slots 4l..4l+3 with one gather; a slot without a row asks for the row behind the
+                // last one, which reads as zeros
+                const int q = (lane & 7) * 4;
+                const uint32_t r0 = __shfl_sync(0xFFFFFFFFu, rows, q), r1 = __shfl_sync(0xFFFFFFFFu, rows, q + 1);
+                const uint32_t r2 = __shfl_sync(0xFFFFFFFFu, rows, q + 2), r3 = __shfl_sync(0xFFFFFFFFu, rows, q + 3);
+                const bool mine = lane < 8 && q < left;  // R is a multiple of 4
+                if (mine)
+                    tma_gather4_rows(stage_base + (uint32_t)((s0 + q) * pitch), &xmap, 0, (int)min(r0, N0), (int)min(r1, N0),
+                                     (int)min(r2, N0), (int)min(r3, N0), full_bar);
+                if (lane < left) {
+                    const bool have = rows != kNoRow;
+                    cp_async_fill<(int)sizeof(T)>(stage_base + (uint32_t)(plan.stage_y_off + (s0 + lane) * (int)sizeof(T)),
+                                                  yb + (have ? rows : 0u), have);
+                }
+                return (uint32_t)__popc(__ballot_sync(0xFFFFFFFFu, mine));
+            } else if constexpr (CB == 16) {
                 const bool have = lane < left && rows != kNoRow;
                 const uint32_t dst = stage_base + (uint32_t)((s0 + lane) * pitch);
                 if (have) {
@@ -582,11 +617,11 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
         };
         // closes this warp's part of a stage: every lane arrives once its element copies have landed, one lane
         // announces the bytes of the warp's bulk copies
-        auto finish_stage = [&](uint32_t full_bar, uint32_t bulk_rows) {
+        auto finish_stage = [&](uint32_t full_bar, uint32_t bulk_rows) {  // bulk_rows: row copies, or gathers of four rows
             mbar_arrive_after_copies(full_bar);
             if constexpr (CB == 16) {
                 __syncwarp();  // the zero fills of all lanes come before the announcing lane's arrival
-                if (lane == 0) mbar_arrive_expect_tx(full_bar, bulk_rows * row_bytes);
+                if (lane == 0) mbar_arrive_expect_tx(full_bar, bulk_rows * (G4 ? (uint32_t)(4 * PCAP * (int)sizeof(T)) : row_bytes));
             }
         };
 
@@ -658,7 +693,9 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
         const uint32_t cpk_base = smem_u32(smem + plan.cpk_off), gpk_base = smem_u32(smem + plan.gpk_off);
         const int lane_off = (warp * GPW + grp) * pitch + sub * CB;  // this lane's first chunk inside a sub-pass
         const int subpass_bytes = spp * pitch;
-        const int y_rel = YOFF - sub * CB;
+        // this group's y in sub-pass 0 of a stage, and how far it moves per sub-pass
+        const int y_off = G4 ? plan.stage_y_off + (warp * GPW + grp) * (int)sizeof(T) : (warp * GPW + grp) * pitch + YOFF;
+        const int y_step = G4 ? spp * (int)sizeof(T) : subpass_bytes;
         const uint32_t warp_first = (uint32_t)(warp * GPW);  // first row slot of this warp in sub-pass 0
         const int slice = (p + S - 1) / S;  // predictors owned by one CTA of a cluster in the sliced exchange
         const T scale_full = (T)P.scale_full, scale_last = (T)P.scale_last;
@@ -694,21 +731,22 @@ __global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1) glm_kernel(
                         bounded_mbar_wait(full_bars + (uint32_t)(cs_slot * 8), cs_phase, aborted, P);
                         __syncwarp();
                         const unsigned char* rowp = smem + plan.ring_off + cs_slot * stage_bytes + lane_off;
+                        const unsigned char* yp = smem + plan.ring_off + cs_slot * stage_bytes + y_off;
                         int nsub = min(sp_left, RB);
                         sp_left -= nsub;
                         if constexpr (NV * (int)sizeof(T) <= 32) {  // narrow rows: four independent rows in flight per group
-                            for (; nsub >= 4; nsub -= 4, rowp += 4 * subpass_bytes) {
-                                row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, y_rel, th, gacc);
-                                row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + subpass_bytes, y_rel, th, gacc);
-                                row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + 2 * subpass_bytes, y_rel, th, gacc);
-                                row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + 3 * subpass_bytes, y_rel, th, gacc);
+                            for (; nsub >= 4; nsub -= 4, rowp += 4 * subpass_bytes, yp += 4 * y_step) {
+                                row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, yp, th, gacc);
+                                row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + subpass_bytes, yp + y_step, th, gacc);
+                                row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + 2 * subpass_bytes, yp + 2 * y_step, th, gacc);
+                                row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + 3 * subpass_bytes, yp + 3 * y_step, th, gacc);
                             }
                         }
-                        for (; nsub >= 2; nsub -= 2, rowp += 2 * subpass_bytes) {  // two independent rows in flight per group
-                            row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, y_rel, th, gacc);
-                            row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + subpass_bytes, y_rel, th, gacc);
+                        for (; nsub >= 2; nsub -= 2, rowp += 2 * subpass_bytes, yp += 2 * y_step) {  // two independent rows in flight per group
+                            row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, yp, th, gacc);
+                            row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + subpass_bytes, yp + y_step, th, gacc);
                         }
-                        if (nsub) row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, y_rel, th, gacc);
+                        if (nsub) row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, yp, th, gacc);
                         __syncwarp();  // every lane has its values in registers: the slot may be refilled
                         if (lane == 0) mbar_arrive(empty_bars + (uint32_t)(cs_slot * 8));
                         if (++cs_slot == D) { cs_slot = 0; cs_phase ^= 1u; }
