@@ -53,6 +53,8 @@ def lib() -> ctypes.CDLL:
             ctypes.c_int, ctypes.c_int, ctypes.c_double, ctypes.c_uint64, ctypes.c_uint32,
             ctypes.c_int, ctypes.c_void_p]
         L.orc_run_rounds.restype = ctypes.c_int
+        L.orc_run_rounds_opt.argtypes = L.orc_run_rounds.argtypes + [ctypes.c_void_p]
+        L.orc_run_rounds_opt.restype = ctypes.c_int
         L.orc_num_threads.restype = ctypes.c_int
         L.orc_set_num_threads.argtypes = [ctypes.c_int]
         _lib = L
@@ -105,7 +107,7 @@ def _as_stored(a):
 
 def run_rounds(loss: int, X, y, theta: np.ndarray, T: int, n: int, alpha: float, seed: int,
                chain: int = 0, C: int = 1, fixed_partition: bool = False,
-               trace: bool = False):
+               trace: bool = False, opt: "Optimizer | None" = None):
     """T rounds over one buffer; `theta` (float64, [p] or [p, C]) is updated in place.
 
     X and y are read as stored (fp64 / fp32 / bf16; int32 labels for softmax).
@@ -130,13 +132,52 @@ def run_rounds(loss: int, X, y, theta: np.ndarray, T: int, n: int, alpha: float,
         raise ValueError("y has the wrong length")
     M = -(-N0 // n)
     tr = np.empty((T * M, theta.size), dtype=np.float64) if trace else None
-    rc = lib().orc_run_rounds(loss, Xn.ctypes.data, xt, yn.ctypes.data, max(yt, 0), N0, p, C,
-                              theta.ctypes.data, T, n, float(alpha),
-                              int(seed) & 0xFFFFFFFFFFFFFFFF, chain, int(fixed_partition),
-                              tr.ctypes.data if trace else None)
+    if opt is not None:
+        if opt.s1.size != theta.size:
+            raise ValueError("optimizer state has the wrong size")
+        st = opt._struct()
+        rc = lib().orc_run_rounds_opt(loss, Xn.ctypes.data, xt, yn.ctypes.data, max(yt, 0), N0, p, C,
+                                      theta.ctypes.data, T, n, float(alpha),
+                                      int(seed) & 0xFFFFFFFFFFFFFFFF, chain, int(fixed_partition),
+                                      tr.ctypes.data if trace else None, ctypes.byref(st))
+    else:
+        rc = lib().orc_run_rounds(loss, Xn.ctypes.data, xt, yn.ctypes.data, max(yt, 0), N0, p, C,
+                                  theta.ctypes.data, T, n, float(alpha),
+                                  int(seed) & 0xFFFFFFFFFFFFFFFF, chain, int(fixed_partition),
+                                  tr.ctypes.data if trace else None)
     if rc != 0:
         raise ValueError("orc_run_rounds rejected its arguments")
     return tr
+
+
+OPT_SGD, OPT_NESTEROV, OPT_ADAM = 0, 1, 2
+LR_CONSTANT, LR_COSINE = 0, 1
+
+
+class _OrcOpt(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int), ("a", ctypes.c_double), ("b", ctypes.c_double), ("eps", ctypes.c_double),
+                ("s1", ctypes.c_void_p), ("s2", ctypes.c_void_p), ("t", ctypes.c_void_p),
+                ("sched", ctypes.c_int), ("period", ctypes.c_int64), ("j_done", ctypes.c_void_p)]
+
+
+class Optimizer:
+    """Update rule and learning-rate schedule with their state, carried from one run_rounds call to the next.
+
+    kind: OPT_SGD (Eq. (2.1)), OPT_NESTEROV (a = momentum) or OPT_ADAM (a = beta1, b = beta2, eps).
+    sched: LR_CONSTANT, or LR_COSINE with `period` updates per pass (Section 4.4).
+    """
+
+    def __init__(self, kind: int, size: int, a: float = 0.9, b: float = 0.999, eps: float = 1e-7,
+                 sched: int = LR_CONSTANT, period: int = 0):
+        self.kind, self.a, self.b, self.eps, self.sched, self.period = kind, a, b, eps, sched, period
+        self.s1 = np.zeros(size, dtype=np.float64)
+        self.s2 = np.zeros(size, dtype=np.float64)
+        self.t = np.zeros(1, dtype=np.int64)
+        self.j_done = np.zeros(1, dtype=np.int64)
+
+    def _struct(self) -> _OrcOpt:
+        return _OrcOpt(self.kind, self.a, self.b, self.eps, self.s1.ctypes.data, self.s2.ctypes.data,
+                       self.t.ctypes.data, self.sched, self.period, self.j_done.ctypes.data)
 
 
 def num_threads() -> int:

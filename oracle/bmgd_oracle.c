@@ -40,9 +40,11 @@
  * bijectivity by brute force; full-batch closed form and OLS limit; the Gram-matrix
  * recurrence Eq. (3.1)-(3.2); the stable solution below Eq. (3.3); tiny-N brute force;
  * finite differences and Newton/IRLS limits for logistic; the C = 2 softmax/logistic
- * identity.  The statistical quality of the shuffle beyond the chi-square gate in the
+ * identity; the Nesterov and Adam updates against a library optimiser fed the same gradients, and against
+ * their closed forms on the first steps; the cosine rate against its printed values.  The statistical quality of the shuffle beyond the chi-square gate in the
  * tests is parity unpinned.
  */
+#define _USE_MATH_DEFINES
 #include <math.h>
 #include <stdint.h>
 #include <stdlib.h>
@@ -50,6 +52,9 @@
 
 #ifdef _OPENMP
 #include <omp.h>
+#endif
+#ifndef M_PI
+#define M_PI 3.14159265358979323846
 #endif
 
 enum { ORC_LINEAR = 0, ORC_LOGISTIC = 1, ORC_SOFTMAX = 2 };
@@ -176,10 +181,89 @@ static double sigmoid(double u) {
  *   trace      if not NULL, receives theta after every step: [T*M][p*C]
  * Returns 0, or -1 on bad arguments.
  */
+enum { ORC_OPT_SGD = 0, ORC_OPT_NESTEROV = 1, ORC_OPT_ADAM = 2 };
+enum { ORC_LR_CONSTANT = 0, ORC_LR_COSINE = 1 };
+
+/*
+ * The update of one step, given the mini-batch's mean gradient g (Section 4.3: "the buffering idea combined
+ * with" other gradient-based rules; the buffered versions differ from their baselines only in where the
+ * mini-batches come from).
+ *
+ *   ORC_OPT_SGD       theta <- theta - lr g                                             Eq. (2.1)
+ *   ORC_OPT_NESTEROV  v <- mu v - lr g;  theta <- theta + mu v - lr g                   (Nesterov's accelerated gradient in
+ *                     the momentum form of Sutskever et al. 2013; mu = a; state s1 = v)
+ *   ORC_OPT_ADAM      m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g^2;  t <- t + 1;
+ *                     theta <- theta - lr (m / (1-b1^t)) / (sqrt(v / (1-b2^t)) + eps)   (Kingma & Ba 2014, Algorithm 1;
+ *                     b1 = a, b2 = b; state s1 = m, s2 = v, *t)
+ *
+ * Learning rate of the j-th update of a pass of J updates (Section 4.4: alpha_{r,j} = 0.025 + 0.025 cos(j pi / TMK)
+ * with initial value 0.05, j = 1..TMK in every pass r):
+ *   ORC_LR_CONSTANT   lr = alpha
+ *   ORC_LR_COSINE     lr = alpha (1/2 + 1/2 cos(j pi / J)),  *j_done counts the updates already taken in this pass
+ */
+typedef struct {
+    int kind;
+    double a, b, eps;
+    double *s1, *s2;   /* [p*C] each, carried from call to call; may be NULL for ORC_OPT_SGD */
+    int64_t *t;        /* Adam's step count, carried from call to call */
+    int sched;
+    int64_t period;    /* J */
+    int64_t *j_done;
+} orc_opt;
+
+static void orc_apply_update(const orc_opt *o, double alpha, int q, const double *gsum, int nm, double *theta) {
+    double lr = alpha;
+    if (o && o->sched == ORC_LR_COSINE) {
+        const int64_t j = *o->j_done + 1;
+        lr = alpha * (0.5 + 0.5 * cos((double)j * M_PI / (double)o->period));
+        *o->j_done = j % o->period;
+    }
+    const int kind = o ? o->kind : ORC_OPT_SGD;
+    if (kind == ORC_OPT_SGD) {
+        const double scale = lr / (double)nm;
+        for (int k = 0; k < q; ++k) theta[k] -= scale * gsum[k];
+    } else if (kind == ORC_OPT_NESTEROV) {
+        for (int k = 0; k < q; ++k) {
+            const double g = gsum[k] / (double)nm;
+            o->s1[k] = o->a * o->s1[k] - lr * g;
+            theta[k] += o->a * o->s1[k] - lr * g;
+        }
+    } else {
+        *o->t += 1;
+        const double c1 = 1.0 - pow(o->a, (double)*o->t), c2 = 1.0 - pow(o->b, (double)*o->t);
+        for (int k = 0; k < q; ++k) {
+            const double g = gsum[k] / (double)nm;
+            o->s1[k] = o->a * o->s1[k] + (1.0 - o->a) * g;
+            o->s2[k] = o->b * o->s2[k] + (1.0 - o->b) * g * g;
+            theta[k] -= lr * (o->s1[k] / c1) / (sqrt(o->s2[k] / c2) + o->eps);
+        }
+    }
+}
+
+int orc_run_rounds_opt(int loss, const void *X, int xtype, const void *y, int ytype,
+                       int64_t N0, int p, int C, double *theta,
+                       int T, int n, double alpha, uint64_t seed, uint32_t chain,
+                       int fixed_partition, double *trace, const orc_opt *opt);
+
 int orc_run_rounds(int loss, const void *X, int xtype, const void *y, int ytype,
                    int64_t N0, int p, int C, double *theta,
                    int T, int n, double alpha, uint64_t seed, uint32_t chain,
                    int fixed_partition, double *trace) {
+    return orc_run_rounds_opt(loss, X, xtype, y, ytype, N0, p, C, theta, T, n, alpha, seed, chain, fixed_partition,
+                              trace, NULL);
+}
+
+/* The same with the update rule and learning-rate schedule of `opt` (NULL: Eq. (2.1) with a constant rate). */
+int orc_run_rounds_opt(int loss, const void *X, int xtype, const void *y, int ytype,
+                       int64_t N0, int p, int C, double *theta,
+                       int T, int n, double alpha, uint64_t seed, uint32_t chain,
+                       int fixed_partition, double *trace, const orc_opt *opt) {
+    if (opt) {
+        if (opt->kind < ORC_OPT_SGD || opt->kind > ORC_OPT_ADAM) return -1;
+        if (opt->kind != ORC_OPT_SGD && !opt->s1) return -1;
+        if (opt->kind == ORC_OPT_ADAM && (!opt->s2 || !opt->t)) return -1;
+        if (opt->sched == ORC_LR_COSINE && (opt->period <= 0 || !opt->j_done)) return -1;
+    }
     if (N0 <= 0 || N0 > 0x7FFFFFFF || p <= 0 || n <= 0 || T < 0) return -1;
     if (loss == ORC_SOFTMAX) { if (C < 2) return -1; } else C = 1;
     const int64_t M = (N0 + n - 1) / n;
@@ -234,8 +318,7 @@ int orc_run_rounds(int loss, const void *X, int xtype, const void *y, int ytype,
                 }
             }
 
-            const double scale = alpha / (double)nm;
-            for (int k = 0; k < q; ++k) theta[k] -= scale * g[k];
+            orc_apply_update(opt, alpha, q, g, nm, theta);
             if (trace) memcpy(trace + (size_t)step * q, theta, sizeof(double) * (size_t)q);
             ++step;
         }
