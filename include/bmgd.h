@@ -198,6 +198,32 @@ int bmgd_get_theta(bmgd_t* h, void* out_host, int64_t bytes);
  * value (Algorithm 1, "Require"), or resuming a run from a saved estimate. */
 int bmgd_set_theta(bmgd_t* h, const void* host, int64_t bytes);
 
+/*
+ * Update rule of the computation step (Section 4.3: the buffering idea "combined with" other gradient-based rules,
+ * BNAG and BAdam beside BMGD; Section 4.2 trains its logistic model with Adam).  With g the mean gradient of the
+ * mini-batch and lr the step's learning rate:
+ *   BMGD_OPT_SGD       theta <- theta - lr g                                   (Eq. (2.1); the default)
+ *   BMGD_OPT_NESTEROV  v <- a v - lr g;  theta <- theta + a v - lr g           (a = momentum, 0 <= a < 1)
+ *   BMGD_OPT_ADAM      m <- a m + (1-a) g;  v <- b v + (1-b) g^2;  t <- t + 1;
+ *                      theta <- theta - lr (m / (1-a^t)) / (sqrt(v / (1-b^t)) + eps)   (Kingma & Ba 2014, Algorithm 1)
+ * The state (v; or m, v and t) lives beside theta on the device, one copy per chain, is carried from call to call
+ * like theta, and is set to zero by this call, which is ordered after the launches already issued.  Linear and
+ * logistic losses; BMGD_ERR_UNIMPLEMENTED for softmax handles.  BMGD_ERR_ARG for values out of range.
+ */
+enum { BMGD_OPT_SGD = 0, BMGD_OPT_NESTEROV = 1, BMGD_OPT_ADAM = 2 };
+int bmgd_set_optimizer(bmgd_t* h, int32_t kind, double a, double b, double eps);
+
+/*
+ * Learning rate of each update (Section 4.4: alpha_{r,j} = 0.025 + 0.025 cos(j pi / TMK) for the j-th update of
+ * every pass r, initial value 0.05).  BMGD_LR_CONSTANT: the lr argument of bmgd_run_rounds, unchanged (the default).
+ * BMGD_LR_COSINE: lr (1/2 + 1/2 cos(j pi / J)) for the j-th update, j = 1..J, of a pass of J = updates_per_pass
+ * updates (T M K in the paper's notation); the count runs on from call to call and starts again after J updates
+ * and when this function is called.  The paper's warm-up has no stated length and is left to the caller (lr is a
+ * per-call argument).  Linear and logistic losses.
+ */
+enum { BMGD_LR_CONSTANT = 0, BMGD_LR_COSINE = 1 };
+int bmgd_set_lr_schedule(bmgd_t* h, int32_t kind, int64_t updates_per_pass);
+
 /* Synchronise and fill *out. */
 int bmgd_get_stats(bmgd_t* h, bmgd_stats* out);
 

@@ -32,7 +32,11 @@ EXPORTS = (
     "bmgd_load_buffer", "bmgd_run_rounds", "bmgd_run_rounds_resident", "bmgd_sync", "bmgd_get_theta",
     "bmgd_set_theta", "bmgd_get_stats", "bmgd_debug_perm", "bmgd_strerror", "bmgd_last_cuda_error",
     "bmgd_version", "bmgd_run_rounds_noalloc", "bmgd_debug_wait_timeout", "bmgd_partition_index", "bmgd_gather_buffer",
+    "bmgd_set_optimizer", "bmgd_set_lr_schedule",
 )
+
+OPT_SGD, OPT_NESTEROV, OPT_ADAM = 0, 1, 2
+LR_CONSTANT, LR_COSINE = 0, 1
 
 
 class BmgdConfig(ctypes.Structure):
@@ -97,6 +101,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.bmgd_run_rounds.argtypes = [vp, i32, i32, i32, dbl, u64]
     L.bmgd_run_rounds_resident.argtypes = [vp, vp, vp, i64, i32, i32, dbl, u64]
     L.bmgd_sync.argtypes = [vp]
+    L.bmgd_set_optimizer.argtypes = [vp, i32, dbl, dbl, dbl]
+    L.bmgd_set_lr_schedule.argtypes = [vp, i32, i64]
     L.bmgd_get_theta.argtypes = [vp, vp, i64]
     L.bmgd_set_theta.argtypes = [vp, vp, i64]
     L.bmgd_get_stats.argtypes = [vp, P(BmgdStats)]
@@ -274,6 +280,15 @@ class Bmgd:
     def set_theta(self, theta: np.ndarray) -> None:
         a = np.ascontiguousarray(theta, dtype=_NP_THETA[self.dtype]).reshape(self.theta_shape)
         self._check(self._lib.bmgd_set_theta(self._h, a.ctypes.data, a.nbytes), "bmgd_set_theta")
+
+    def set_optimizer(self, kind: int, a: float = 0.0, b: float = 0.0, eps: float = 0.0) -> None:
+        """Choose the update rule (OPT_SGD, OPT_NESTEROV with momentum a, OPT_ADAM with beta1 a, beta2 b, eps);
+        its state starts from zero."""
+        self._check(self._lib.bmgd_set_optimizer(self._h, kind, float(a), float(b), float(eps)), "bmgd_set_optimizer")
+
+    def set_lr_schedule(self, kind: int, updates_per_pass: int = 0) -> None:
+        """LR_CONSTANT, or LR_COSINE: the j-th update of a pass of `updates_per_pass` takes lr (1/2 + 1/2 cos(j pi / J))."""
+        self._check(self._lib.bmgd_set_lr_schedule(self._h, kind, int(updates_per_pass)), "bmgd_set_lr_schedule")
 
     def get_stats(self) -> dict:
         st = BmgdStats()

@@ -46,7 +46,7 @@ struct EventPair {
 
 struct Layout {
     int64_t slot_x[2], slot_y[2];
-    int64_t theta, ll, status, softmax_scratch;
+    int64_t theta, opt1, opt2, ll, status, softmax_scratch;
     int64_t total;
 };
 
@@ -75,6 +75,13 @@ struct bmgd {
     bmgd_stats stats{};
     std::vector<EventPair> kernel_events, copy_events, event_pool;
     uint64_t timeout_ns = 2000000000ull;
+    // update rule and learning-rate schedule (bmgd_set_optimizer, bmgd_set_lr_schedule)
+    int opt_kind = BMGD_OPT_SGD;
+    double opt_a = 0.0, opt_b = 0.0, opt_eps = 0.0;
+    int64_t opt_steps = 0;     // updates taken since the rule was set: Adam's t
+    int sched = BMGD_LR_CONSTANT;
+    int64_t sched_period = 0;  // updates per pass
+    int64_t sched_pos = 0;     // updates of the current pass already taken
 };
 
 namespace {
@@ -140,6 +147,9 @@ Layout make_layout(const bmgd_config* c) {
         L.slot_y[s] = off; if (s < slots) off += align_up(N0 * yb);
     }
     L.theta = off; off += align_up((int64_t)c->Rc * c->p * c->C * tb);
+    // state of the update rule, beside theta: Nesterov's velocity or Adam's first moment, and Adam's second moment
+    L.opt1 = off; if (c->loss != BMGD_LOSS_SOFTMAX) off += align_up((int64_t)c->Rc * c->p * tb);
+    L.opt2 = off; if (c->loss != BMGD_LOSS_SOFTMAX) off += align_up((int64_t)c->Rc * c->p * tb);
     L.ll = off;
     if (c->loss != BMGD_LOSS_SOFTMAX) off += align_up((int64_t)2 * kMaxClustersForExchange * c->p * 2 * 8);
     L.status = off; off += kAlign;
@@ -278,8 +288,9 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     if (S == 0) {
         if (c.Rc > 1) S = std::min(8, floor_pow2(std::max(1, h->sm_count / c.Rc)));
         else S = 16;
-        // do not spread a mini-batch thinner than 8 rows per CTA
-        while (S > 1 && n / S < 8) S /= 2;
+        // do not spread a mini-batch thinner than one sweep of a CTA over its rows: below that a larger cluster only
+        // adds exchange latency (measured on B200: n = 100 runs fastest on 2 CTAs)
+        while (S > 1 && n / S < spp) S /= 2;
     }
 
     // How many clusters can be resident depends on shared memory, which depends on the ring; ask with
@@ -421,6 +432,14 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
     P.timeout_ns = h->timeout_ns;
     P.scale_full = lr / (double)n;
     P.scale_last = lr / (double)(rows - (int64_t)(M - 1) * n);
+    P.lr = lr;
+    P.inv_full = 1.0 / (double)n;
+    P.inv_last = 1.0 / (double)(rows - (int64_t)(M - 1) * n);
+    P.opt1 = h->base + h->lay.opt1; P.opt2 = h->base + h->lay.opt2;
+    P.opt_kind = h->opt_kind; P.opt_a = h->opt_a; P.opt_b = h->opt_b; P.opt_eps = h->opt_eps;
+    P.adam_b1pow0 = std::pow(h->opt_a, (double)h->opt_steps);
+    P.adam_b2pow0 = std::pow(h->opt_b, (double)h->opt_steps);
+    P.sched = h->sched; P.sched_period = h->sched_period; P.sched_pos0 = h->sched_pos;
     P.N0 = (uint32_t)rows; P.n = (uint32_t)n; P.M = M; P.T = rounds; P.p = c.p;
     P.Rc = c.Rc; P.S = L.S; P.cpc = L.cpc; P.nteams = L.nteams;
     P.passes = L.passes; P.rb = L.rb; P.depth = L.depth;
@@ -479,6 +498,8 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
         h->kernel_events.push_back(ep);
     }
     h->tag_base += steps_per_team;
+    h->opt_steps += (int64_t)rounds * M;
+    if (h->sched == BMGD_LR_COSINE) h->sched_pos = (h->sched_pos + (int64_t)rounds * M) % h->sched_period;
     h->stats.launches += 1;
     h->stats.steps += (int64_t)c.Rc * rounds * M;
     h->stats.sample_grads += (int64_t)c.Rc * rounds * rows;
@@ -742,6 +763,32 @@ int bmgd_set_theta(bmgd_t* h, const void* host, int64_t bytes) {
     return BMGD_OK;
 }
 
+int bmgd_set_optimizer(bmgd_t* h, int32_t kind, double a, double b, double eps) {
+    if (!h) return BMGD_ERR_ARG;
+    if (kind < BMGD_OPT_SGD || kind > BMGD_OPT_ADAM) return BMGD_ERR_ARG;
+    if (kind == BMGD_OPT_NESTEROV && !(a >= 0.0 && a < 1.0)) return BMGD_ERR_ARG;
+    if (kind == BMGD_OPT_ADAM && !(a >= 0.0 && a < 1.0 && b >= 0.0 && b < 1.0 && eps > 0.0)) return BMGD_ERR_ARG;
+    if (h->cfg.loss == BMGD_LOSS_SOFTMAX) return kind == BMGD_OPT_SGD ? BMGD_OK : BMGD_ERR_UNIMPLEMENTED;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return cuda_fail(h, cudaErrorInvalidDevice);
+    // the state starts from zero, ordered after the launches already issued
+    BMGD_CUDA(h, cudaMemsetAsync(h->base + h->lay.opt1, 0, (size_t)(h->lay.ll - h->lay.opt1), h->compute));
+    h->opt_kind = kind; h->opt_a = a; h->opt_b = b; h->opt_eps = eps;
+    h->opt_steps = 0;
+    return BMGD_OK;
+}
+
+int bmgd_set_lr_schedule(bmgd_t* h, int32_t kind, int64_t updates_per_pass) {
+    if (!h) return BMGD_ERR_ARG;
+    if (kind != BMGD_LR_CONSTANT && kind != BMGD_LR_COSINE) return BMGD_ERR_ARG;
+    if (kind == BMGD_LR_COSINE && updates_per_pass <= 0) return BMGD_ERR_ARG;
+    if (h->cfg.loss == BMGD_LOSS_SOFTMAX) return kind == BMGD_LR_CONSTANT ? BMGD_OK : BMGD_ERR_UNIMPLEMENTED;
+    h->sched = kind;
+    h->sched_period = kind == BMGD_LR_COSINE ? updates_per_pass : 0;
+    h->sched_pos = 0;
+    return BMGD_OK;
+}
+
 int bmgd_get_stats(bmgd_t* h, bmgd_stats* out) {
     if (!h || !out) return BMGD_ERR_ARG;
     DeviceGuard guard(h->device);
@@ -861,6 +908,10 @@ int bmgd_run_rounds_noalloc(const void* dev_x, const void* dev_y, int64_t rows, 
     P.timeout_ns = 2000000000ull;
     P.scale_full = lr / (double)n;
     P.scale_last = lr / (double)(rows - (int64_t)(M - 1) * n);
+    P.lr = lr;
+    P.inv_full = 1.0 / (double)n;
+    P.inv_last = 1.0 / (double)(rows - (int64_t)(M - 1) * n);
+    P.opt_kind = bmgdk::kOptSgd; P.sched = bmgdk::kLrConstant;  // Eq. (2.1) with a constant rate: no state beside theta
     P.N0 = (uint32_t)rows; P.n = (uint32_t)n; P.M = M; P.T = rounds; P.p = p;
     P.Rc = Rc; P.S = L.S; P.cpc = L.cpc; P.nteams = L.nteams;
     P.passes = L.passes; P.rb = L.rb; P.depth = L.depth;

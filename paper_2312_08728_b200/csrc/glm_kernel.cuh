@@ -19,8 +19,11 @@
 //      packets that arrive in its own.  With several clusters the partials are reduce-scattered inside the
 //      cluster the same way (CTA r owns a slice of the predictors), the slice sums cross clusters as tagged
 //      packets in global memory (only the slice owner polls), and the totals are pushed to every peer;
-//   4. every CTA applies theta <- theta - (alpha/n_m) g to its own register copy of theta.
-// All sums have a fixed order, so all CTAs hold bit-identical theta and runs are reproducible.
+//   4. in every CTA the thread that holds predictor f's total applies the update rule (Eq. (2.1); or Nesterov's or
+//      Adam's, Section 4.3; with a constant or a per-update cosine rate, Section 4.4) to its master copy of theta_f
+//      and the lanes reload the coefficients they multiply rows with.
+// All sums have a fixed order and every CTA does the same arithmetic, so all CTAs hold bit-identical theta and runs
+// are reproducible.
 //
 // Every wait on another warp or CTA is bounded: when the budget runs out the kernel records
 // BMGD_ERR_TIMEOUT in the status word, stops waiting for the rest of the launch and returns.
@@ -37,6 +40,8 @@ constexpr int kMaxCpc = 20;        // clusters per chain the packet exchange is 
 constexpr int kMaxClusterSize = 16; // CTAs per cluster
 constexpr int kMaxBatchesPerProducer = 2;  // batches of 32 row slots one producer warp takes in one ring stage
 constexpr int kStatusTimeout = -5; // == BMGD_ERR_TIMEOUT
+constexpr int kOptSgd = 0, kOptNesterov = 1, kOptAdam = 2;  // == BMGD_OPT_*
+constexpr int kLrConstant = 0, kLrCosine = 1;               // == BMGD_LR_*
 
 struct GlmParams {
     const void* X;        // [N0][p] rows
@@ -48,6 +53,15 @@ struct GlmParams {
     unsigned long long timeout_ns;
     double scale_full;    // alpha / n: step size over a full mini-batch
     double scale_last;    // alpha / (size of the ragged last mini-batch of a round)
+    double lr;            // alpha
+    double inv_full, inv_last;  // 1 / n and 1 / (size of the last mini-batch)
+    void* opt1;           // update-rule state [Rc][p]: Nesterov's velocity, Adam's first moment
+    void* opt2;           // Adam's second moment [Rc][p]
+    double opt_a, opt_b, opt_eps;        // momentum; or beta1, beta2, epsilon
+    double adam_b1pow0, adam_b2pow0;     // beta1^t, beta2^t after the steps taken by earlier calls
+    long long sched_period, sched_pos0;  // cosine rate: updates per pass, and how many of this pass are done
+    int opt_kind;         // kOptSgd / kOptNesterov / kOptAdam
+    int sched;            // kLrConstant / kLrCosine
     uint32_t N0;
     uint32_t n;           // mini-batch size
     uint32_t M;           // mini-batches per round
@@ -699,6 +713,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
         const uint32_t warp_first = (uint32_t)(warp * GPW);  // first row slot of this warp in sub-pass 0
         const int slice = (p + S - 1) / S;  // predictors owned by one CTA of a cluster in the sliced exchange
         const T scale_full = (T)P.scale_full, scale_last = (T)P.scale_last;
+        const T inv_full = (T)P.inv_full, inv_last = (T)P.inv_last, lr_const = (T)P.lr;
 
         int cs_slot = 0;         // ring slot the compute cursor reads next
         uint32_t cs_phase = 0;   // parity of that slot's "full" phase
@@ -715,6 +730,19 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
 #pragma unroll
                 for (int e = 0; e < VEC; ++e) th[k * VEC + e] = (c < nchunks) ? theta_g[c * VEC + e] : T(0);
             }
+            // thread f's master copy of theta_f and the update rule's state for it (velocity; or first and second moment)
+            T thm[FPT], st1[FPT], st2[FPT];
+            T* st1_g = static_cast<T*>(P.opt1) + (size_t)chain * p;
+            T* st2_g = static_cast<T*>(P.opt2) + (size_t)chain * p;
+#pragma unroll
+            for (int i = 0; i < FPT; ++i) {
+                const int f = tid + i * nthreads;
+                thm[i] = (f < p) ? theta_g[f] : T(0);
+                st1[i] = (f < p && P.opt_kind != kOptSgd) ? st1_g[f] : T(0);
+                st2[i] = (f < p && P.opt_kind == kOptAdam) ? st2_g[f] : T(0);
+            }
+            double b1pow = P.adam_b1pow0, b2pow = P.adam_b2pow0;  // beta^t after the steps of earlier calls
+            long long sched_pos = P.sched_pos0;                   // updates already taken in this pass
 
             for (int t = 0; t < T_rounds; ++t) {
                 for (uint32_t m = 0; m < M; ++m) {
@@ -817,12 +845,6 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                         }
                         BMGD_STAMP(4);
                         BMGD_STAMP(5);
-    #pragma unroll
-                        for (int i = 0; i < FPT; ++i) {
-                            const int f = tid + i * nthreads;
-                            if (f < p) gfin[f] = tot[i];
-                        }
-                        consumer_sync(nthreads);
                     } else {
                         // ---- several clusters per chain: reduce-scatter in the cluster (CTA r owns a slice of the
                         //      predictors and receives its peers' partial sums as tagged packets), packets through global
@@ -879,7 +901,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                                     for (int peer = 0; peer < S; ++peer) st_cluster_u64(map_to_cta(dst, (uint32_t)peer), pk);
                                 }
                             } else {
-                                gfin[f] = s;
+                                tot[i] = s;  // one CTA per cluster: j == f
                             }
                         }
                         BMGD_STAMP(5);
@@ -888,31 +910,70 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                             for (int i = 0; i < FPT; ++i) {
                                 const int f = tid + i * nthreads;
                                 if (f < p)
-                                    gfin[f] = gather_packets<T, 1, 1>(
+                                    tot[i] = gather_packets<T, 1, 1>(
                                         1, tag, aborted, P,
                                         [&](int, int w) { return ld_shared_volatile_u64(gpk + (uint32_t)((f * NW + w) * 8)); });
                             }
                         }
-                        consumer_sync(nthreads);
                     }
                     BMGD_STAMP(6);
 
-                    // ---- everyone updates its own copy of theta
-                    const T scale = (min(n, N0 - sh.lo) == n) ? scale_full : scale_last;
+                    // ---- the thread that holds predictor f's gradient sum applies the update rule to its master copy of
+                    //      theta_f (the same arithmetic in every CTA, so all copies stay bit-identical) and publishes it;
+                    //      then every lane refreshes the coefficients it multiplies rows with
+                    const bool full = min(n, N0 - sh.lo) == n;
+                    T lr = lr_const;
+                    if (P.sched == kLrCosine) {  // Section 4.4: rate of the j-th update of a pass of J updates
+                        const long long j = sched_pos + 1;
+                        lr = (T)(P.lr * (0.5 + 0.5 * cospi((double)j / (double)P.sched_period)));
+                        sched_pos = (j == P.sched_period) ? 0 : j;
+                    }
+                    if (P.opt_kind == kOptSgd) {
+                        const T scale = (P.sched == kLrCosine) ? lr * (full ? inv_full : inv_last) : (full ? scale_full : scale_last);
+#pragma unroll
+                        for (int i = 0; i < FPT; ++i) {
+                            const int f = tid + i * nthreads;
+                            if (f < p) { thm[i] = fma(-scale, tot[i], thm[i]); gfin[f] = thm[i]; }
+                        }
+                    } else if (P.opt_kind == kOptNesterov) {
+                        const T inv = full ? inv_full : inv_last, mu = (T)P.opt_a;
+#pragma unroll
+                        for (int i = 0; i < FPT; ++i) {
+                            const int f = tid + i * nthreads;
+                            if (f < p) {
+                                const T gm = tot[i] * inv;
+                                st1[i] = mu * st1[i] - lr * gm;
+                                thm[i] = thm[i] + mu * st1[i] - lr * gm;
+                                gfin[f] = thm[i];
+                            }
+                        }
+                    } else {  // Adam
+                        const T inv = full ? inv_full : inv_last, b1 = (T)P.opt_a, b2 = (T)P.opt_b, eps = (T)P.opt_eps;
+                        b1pow *= P.opt_a; b2pow *= P.opt_b;  // beta^t, in double
+                        const T c1 = (T)(1.0 - b1pow), c2 = (T)(1.0 - b2pow);
+#pragma unroll
+                        for (int i = 0; i < FPT; ++i) {
+                            const int f = tid + i * nthreads;
+                            if (f < p) {
+                                const T gm = tot[i] * inv;
+                                st1[i] = b1 * st1[i] + (T(1) - b1) * gm;
+                                st2[i] = b2 * st2[i] + (T(1) - b2) * gm * gm;
+                                thm[i] = thm[i] - lr * (st1[i] / c1) / (sqrt(st2[i] / c2) + eps);
+                                gfin[f] = thm[i];
+                            }
+                        }
+                    }
+                    consumer_sync(nthreads);
                     {
                         const T* gf = gfin + sub * VEC;
 #pragma unroll
                         for (int k = 0; k < KCH; ++k) {
                             if constexpr (CB == 16 && sizeof(T) == 4) {
                                 const float4 v = *reinterpret_cast<const float4*>(gf + k * LPR * VEC);
-                                th[k * VEC + 0] = fma(-scale, v.x, th[k * VEC + 0]);
-                                th[k * VEC + 1] = fma(-scale, v.y, th[k * VEC + 1]);
-                                th[k * VEC + 2] = fma(-scale, v.z, th[k * VEC + 2]);
-                                th[k * VEC + 3] = fma(-scale, v.w, th[k * VEC + 3]);
+                                th[k * VEC + 0] = v.x; th[k * VEC + 1] = v.y; th[k * VEC + 2] = v.z; th[k * VEC + 3] = v.w;
                             } else {
 #pragma unroll
-                                for (int e = 0; e < VEC; ++e)
-                                    th[k * VEC + e] = fma(-scale, gf[k * LPR * VEC + e], th[k * VEC + e]);
+                                for (int e = 0; e < VEC; ++e) th[k * VEC + e] = gf[k * LPR * VEC + e];
                             }
                         }
                     }
@@ -921,13 +982,15 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                 }
             }
 
-            if (g == 0 && warp == 0 && grp == 0) {
+            if (g == 0) {
 #pragma unroll
-                for (int k = 0; k < KCH; ++k) {
-                    const int c = sub + k * LPR;
-                    if (c < nchunks)
-#pragma unroll
-                        for (int e = 0; e < VEC; ++e) theta_g[c * VEC + e] = th[k * VEC + e];
+                for (int i = 0; i < FPT; ++i) {
+                    const int f = tid + i * nthreads;
+                    if (f < p) {
+                        theta_g[f] = thm[i];
+                        if (P.opt_kind != kOptSgd) st1_g[f] = st1[i];
+                        if (P.opt_kind == kOptAdam) st2_g[f] = st2[i];
+                    }
                 }
             }
         }

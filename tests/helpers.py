@@ -16,23 +16,31 @@ def rel_l2(a, b):
     return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
 
 
-def oracle_job(w, buffers, chains=None, theta0=None, fixed_partition=False):
-    """Run w.epochs passes over `buffers` [(X, y), ...] for the listed chains; returns {chain: theta}."""
+def oracle_job(w, buffers, chains=None, theta0=None, fixed_partition=False, opt=None):
+    """Run w.epochs passes over `buffers` [(X, y), ...] for the listed chains; returns {chain: theta}.
+
+    opt: None, or dict(kind=, a=, b=, eps=, sched=, period=) in the oracle's constants: the update rule and
+    learning-rate schedule, with one state per chain carried through the whole job."""
     chains = list(range(w.Rc)) if chains is None else chains
     shape = (w.p, w.C) if w.loss == inputs.LOSS_SOFTMAX else (w.p,)
     out = {}
     for c in chains:
         th = np.zeros(shape) if theta0 is None else np.array(theta0[c], dtype=np.float64).reshape(shape)
+        o = None
+        if opt is not None:
+            o = oracle.Optimizer(opt.get("kind", oracle.OPT_SGD), th.size, a=opt.get("a", 0.0), b=opt.get("b", 0.0),
+                                 eps=opt.get("eps", 0.0), sched=opt.get("sched", oracle.LR_CONSTANT),
+                                 period=opt.get("period", 0))
         for e in range(w.epochs):
             for k, (X, y) in enumerate(buffers):
                 oracle.run_rounds(ORACLE_LOSS[w.loss], X, y, th, w.T, min(w.n, X.shape[0]), w.lr,
                                   inputs.buffer_seed(w.seed, e, k, len(buffers)), chain=c, C=w.C,
-                                  fixed_partition=fixed_partition)
+                                  fixed_partition=fixed_partition, opt=o)
         out[c] = th
     return out
 
 
-def gpu_job(w, buffers, mode="slots", flags=0, theta0=None, **shape):
+def gpu_job(w, buffers, mode="slots", flags=0, theta0=None, opt=None, **shape):
     """The same job through the C ABI.  mode: "slots" streams host buffers through load_buffer with the next
     copy issued before the current compute; "resident" keeps all buffers on the device."""
     from paper_2312_08728_b200.binding import Bmgd, FLAG_NO_SLOTS
@@ -44,6 +52,9 @@ def gpu_job(w, buffers, mode="slots", flags=0, theta0=None, **shape):
     try:
         if theta0 is not None:
             h.set_theta(theta0)
+        if opt is not None:  # the library's constants have the oracle's values; checked in the CPU tests
+            h.set_optimizer(opt.get("kind", 0), opt.get("a", 0.0), opt.get("b", 0.0), opt.get("eps", 0.0))
+            h.set_lr_schedule(opt.get("sched", 0), opt.get("period", 0))
         if mode == "resident":
             dev = [(X.cuda(), y.cuda()) for X, y in buffers]
             for e in range(w.epochs):
