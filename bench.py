@@ -241,8 +241,8 @@ def config_of(args, w):
                         f"n={w.n}, T={w.T}, lr={w.lr}, Rc={w.Rc}" + (f", C={w.C}" if w.C > 1 else ""),
             "step": "one buffer: T rounds x M mini-batch steps x Rc chains in one launch",
             "cache": "steps cycle through the workload's buffers; the buffer set is larger than L2 "
-                     "(a single buffer of cfg2 is not: its 640 re-reads per step are served by L2 by design)"
-                     if w.name == "cfg2" else "steps cycle through the workload's buffers; inputs larger than L2"}
+                     f"(a single buffer is not: its Rc*T = {w.Rc * w.T} re-reads per step are served by L2 by design)"
+                     if w.Rc > 1 else "steps cycle through the workload's buffers; inputs larger than L2"}
 
 
 # ---------------------------------------------------------------------------------------------- our arm
@@ -375,9 +375,10 @@ def run_ours(args, w):
         roofline["tensor_tflops"] = flops / kdur / 1e12 if kdur > 0 else None
         roofline["note"] = ("bf16 tcgen05 contractions (M=128, N=16, K=16); the step is bound by its two cluster "
                             "barriers and the gather, not by the tensor pipe or HBM")
-    if w.name == "cfg2":
-        roofline["note"] = ("one 40 MB buffer is re-read Rc*T = 640 times per launch and stays in the 126 MB L2, "
-                            "so algorithmic bytes per second may exceed the HBM peak; DRAM traffic is in `traffic`")
+    if w.Rc > 1:
+        roofline["note"] = (f"one {w.N0 * w.p * w.x_itemsize / 1e6:.0f} MB buffer is re-read Rc*T = {w.Rc * w.T} times per launch "
+                            "and stays in the 126 MB L2, so algorithmic bytes per second may exceed the HBM peak; "
+                            "DRAM traffic is in `traffic`")
 
     cpu = None
     if not args.no_cpu and world == 1:

@@ -53,6 +53,7 @@ class Workload:
     C: int = 1      # classes (softmax only)
     rho: float = 0.0
     seed: int = 0
+    design: str = ""  # "unit-signal": theta* drawn standard normal and scaled so that var(x.theta*) = 1
 
     @property
     def N0(self) -> int:
@@ -101,6 +102,11 @@ WORKLOADS = {
                      epochs=2, C=10, seed=0),
     "cfg5": Workload("cfg5", LOSS_LINEAR, DTYPE_F32, N=50_000_000, p=64, K=20, n=2_048, T=5, lr=0.01,
                      epochs=1, rho=0.5, seed=0),
+    # The shape of the paper's own linear simulation (Section 4.1): N = 100,000, p = 500, Sigma = 0.8^|i-j|, unit signal
+    # variance, buffers of 10,000, mini-batches of 1,000, T = 5 with alpha T = 0.01, 100 passes, 100 replicates.  Here the
+    # replicates are chains over one data set with their own shuffles; the paper redraws the data for each.
+    "sim41": Workload("sim41", LOSS_LINEAR, DTYPE_F32, N=100_000, p=500, K=10, n=1_000, T=5, lr=0.002,
+                      epochs=100, Rc=100, rho=0.8, seed=41, design="unit-signal"),
 }
 
 
@@ -127,6 +133,12 @@ def _ar_rows(rows: int, p: int, rho: float, g: torch.Generator) -> torch.Tensor:
 
 def theta_star(w: Workload) -> torch.Tensor:
     """True coefficients of the generating model, fp64; [p] or [p, C]."""
+    if w.design == "unit-signal":
+        # the paper's simulation design (Section 4.1): theta* ~ N(0, I), then scaled so that theta*' Sigma theta* = 1
+        z = torch.randn(w.p, generator=_gen(w.seed, 1), dtype=torch.float64)
+        idx = torch.arange(w.p, dtype=torch.float64)
+        sigma = w.rho ** (idx[:, None] - idx[None, :]).abs() if w.rho != 0.0 else torch.eye(w.p, dtype=torch.float64)
+        return z / torch.sqrt(z @ sigma @ z)
     if w.loss == LOSS_LINEAR:
         return torch.ones(w.p, dtype=torch.float64)
     if w.loss == LOSS_LOGISTIC:

@@ -213,6 +213,13 @@ def test_cfg3_one_full_buffer_default_shape():
     check(w, buffers_of(w), mode="resident")
 
 
+def test_cfg5_one_full_buffer_default_shape():
+    """One full cfg5 buffer (2,500,000 x 64, n=2,048: 1,221 steps per round with a ragged last one), through a slot."""
+    w = WORKLOADS["cfg5"].scaled(N=2_500_000, K=1, T=2, epochs=1)
+    _, stats, _ = check(w, buffers_of(w), mode="slots")
+    assert stats["steps"] == 2 * 1221
+
+
 def test_a_wait_that_runs_out_is_reported_and_the_handle_stays_usable():
     """Failure detection without a GPU fault: a bounded wait gives up after its budget, the status word carries
     BMGD_ERR_TIMEOUT to the next synchronising call, and the same handle then computes correctly."""
