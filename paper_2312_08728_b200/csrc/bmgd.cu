@@ -202,7 +202,9 @@ int make_row_map(const void* dev_x, int64_t rows, int p, int elem_bytes, int box
 typedef void (*GlmKernel)(const GlmParams, const CUtensorMap);
 
 struct GlmVariant {
-    GlmKernel fn;
+    GlmKernel fn_small;  // compiled for CTAs of up to kGlmSmallCta threads (more registers per thread)
+    GlmKernel fn_large;  // compiled for CTAs of up to kGlmLargeCta threads, or null
+    GlmKernel fn(int cta_threads) const { return (cta_threads > bmgdk::kGlmSmallCta && fn_large) ? fn_large : fn_small; }
     int vec, lpr, kch, maxc, maxt;
     int cap() const { return vec * lpr * kch; }
     int max_consumer_threads() const { return maxc; }  // warps that compute
@@ -212,7 +214,10 @@ struct GlmVariant {
 template <typename T, bool LG>
 const GlmVariant* glm_variants(bool aligned16, int* count) {
     constexpr int V = 16 / (int)sizeof(T);
-#define BMGD_VAR(VEC, LPR, KCH) {bmgdk::glm_kernel<T, VEC, LPR, KCH, LG>, VEC, LPR, KCH, \
+#define BMGD_VAR(VEC, LPR, KCH) {bmgdk::glm_kernel<T, VEC, LPR, KCH, LG, bmgdk::kGlmSmallCta>, \
+                                 (bmgdk::glm_max_threads<T, VEC, KCH>() != bmgdk::kGlmSmallCta) \
+                                     ? bmgdk::glm_kernel<T, VEC, LPR, KCH, LG, bmgdk::glm_max_threads<T, VEC, KCH>()> : nullptr, \
+                                 VEC, LPR, KCH, \
                                  bmgdk::glm_max_consumer_threads<T, VEC, KCH>(), bmgdk::glm_max_threads<T, VEC, KCH>()}
     static const GlmVariant wide[] = {BMGD_VAR(V, 8, 1), BMGD_VAR(V, 8, 2), BMGD_VAR(V, 8, 4),
                                       BMGD_VAR(V, 8, 8), BMGD_VAR(V, 16, 8), BMGD_VAR(V, 32, 8)};
@@ -304,11 +309,11 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
             return BMGD_ERR_UNIMPLEMENTED;
         }
         const int probe_smem = fixed_smem + ring_budget;
-        BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn, cudaFuncAttributeMaxDynamicSharedMemorySize, probe_smem));
-        BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn, cudaFuncAttributeNonPortableClusterSizeAllowed, S > 8 ? 1 : 0));
+        BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn(L.threads + 32 * L.pwarps), cudaFuncAttributeMaxDynamicSharedMemorySize, probe_smem));
+        BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn(L.threads + 32 * L.pwarps), cudaFuncAttributeNonPortableClusterSizeAllowed, S > 8 ? 1 : 0));
         max_clusters = h->sm_count;
         if (S > 1) {
-            int rc = max_active_clusters(h, var->fn, S, L.threads + 32 * L.pwarps, probe_smem, &max_clusters);
+            int rc = max_active_clusters(h, var->fn(L.threads + 32 * L.pwarps), S, L.threads + 32 * L.pwarps, probe_smem, &max_clusters);
             if (rc != BMGD_OK) {
                 if (c.cluster_size == 0 && S > 8) { S = 8; continue; }  // clusters of 16 are optional in hardware
                 return rc;
@@ -485,7 +490,7 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
             return rc;
         }
     }
-    cudaError_t e = cudaLaunchKernelEx(&lc, var->fn, P, xmap);
+    cudaError_t e = cudaLaunchKernelEx(&lc, var->fn(L.threads + 32 * L.pwarps), P, xmap);
     if (e != cudaSuccess) {
         h->last_cuda = (int)e;
         cudaGetLastError();
@@ -945,7 +950,7 @@ int bmgd_run_rounds_noalloc(const void* dev_x, const void* dev_y, int64_t rows, 
         rc = make_row_map(dev_x, rows, p, tb, var->cap(), &xmap);
         if (rc != BMGD_OK) return rc;
     }
-    cudaError_t e = cudaLaunchKernelEx(&lc, var->fn, P, xmap);
+    cudaError_t e = cudaLaunchKernelEx(&lc, var->fn(L.threads + 32 * L.pwarps), P, xmap);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return (e == cudaErrorCooperativeLaunchTooLarge || e == cudaErrorLaunchOutOfResources) ? BMGD_ERR_LAUNCH : BMGD_ERR_CUDA;

@@ -93,7 +93,6 @@ __device__ __forceinline__ void cp_async(uint32_t dst_smem, const void* src) {
     else
         asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst_smem), "l"(src) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 // One chunk of BYTES bytes: copied from `src` if `have`, otherwise written as zeros (nothing is read from `src`).
 template <int BYTES>
@@ -118,14 +117,8 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t cta)
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(cta));
     return r;
 }
-__device__ __forceinline__ void st_cluster(uint32_t addr, float v) {
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
-}
 __device__ __forceinline__ void st_shared_zero16(uint32_t addr) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0) : "memory");
-}
-__device__ __forceinline__ void st_cluster(uint32_t addr, double v) {
-    asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(addr), "d"(v) : "memory");
 }
 // A 64-bit store into a peer's shared memory and a re-read of one's own: value and tag travel together.
 __device__ __forceinline__ void st_cluster_u64(uint32_t addr, unsigned long long v) {
@@ -282,12 +275,13 @@ template <typename T, int VEC, int KCH>
 __host__ __device__ constexpr int glm_max_consumer_threads() {
     return (sizeof(T) == 8 || KCH * VEC >= 32) ? 256 : 512;
 }
-#ifndef BMGD_GLM_MAX_THREADS
-#define BMGD_GLM_MAX_THREADS 640
-#endif
+// CTA sizes a kernel is compiled for (consumers plus producers; registers come in units of four warps): kGlmSmallCta
+// leaves 168 registers per thread, kGlmLargeCta 96 and is built only for variants with little per-lane state.  (A
+// 512-thread instance with 128 registers was measured too: never the fastest.)
+constexpr int kGlmSmallCta = 256 + 128, kGlmLargeCta = 512 + 128;
 template <typename T, int VEC, int KCH>
 __host__ __device__ constexpr int glm_max_threads() {
-    return (sizeof(T) == 8 || KCH * VEC >= 32) ? 256 + 128 : BMGD_GLM_MAX_THREADS;  // registers come in units of four warps
+    return (sizeof(T) == 8 || KCH * VEC >= 32) ? kGlmSmallCta : kGlmLargeCta;
 }
 // Few values per lane: fold the row groups of a warp together by shuffles before shared memory.
 template <int VEC, int KCH>
@@ -471,8 +465,8 @@ __device__ __forceinline__ void bounded_mbar_wait(uint32_t bar, uint32_t parity,
 // row beyond p is zeroed once and never written, and a slot without a row is zero-filled by its copy, so the
 // inner loop carries no predicates.  Each stage has a "full" mbarrier (the producers' copies have landed) and an
 // "empty" one (every consumer warp has read it).
-template <typename T, int VEC, int LPR, int KCH, bool LOGISTIC>
-__global__ void __launch_bounds__(glm_max_threads<T, VEC, KCH>(), 1)
+template <typename T, int VEC, int LPR, int KCH, bool LOGISTIC, int MAXT>
+__global__ void __launch_bounds__(MAXT, 1)
 glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
     constexpr int GPW = 32 / LPR;            // row groups per warp
     constexpr int NV = KCH * VEC;            // values per lane
