@@ -828,6 +828,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                                     }
                                 }
                             }
+                            BMGD_STAMP(8);
     #pragma unroll
                             for (int i = 0; i < FPT; ++i) {
                                 const int f = tid + i * nthreads;
@@ -957,6 +958,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                             }
                         }
                     }
+                    BMGD_STAMP(9);
                     consumer_sync(nthreads);
                     {
                         const T* gf = gfin + sub * VEC;
