@@ -303,7 +303,7 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     int max_clusters = 0, fixed_smem = 0, ring_budget = 0;
     for (;;) {
         fixed_smem = bmgdk::glm_smem_plan(warps, gpw, pre, 1, 0, pcap, eb, S, false, gathered).total_bytes;
-        ring_budget = std::min(h->smem_optin - fixed_smem, 160 * 1024);
+        ring_budget = h->smem_optin - fixed_smem - 1024;  // all of the CTA's shared memory but a small reserve
         if (ring_budget < 2 * bmgdk::glm_smem_plan(warps, gpw, pre, 1, 1, pcap, eb, S, false, gathered).stage_bytes) {  // the per-peer exchange buffers of a large cluster leave no room for rows
             if (c.cluster_size == 0 && S > 1) { S /= 2; continue; }
             return BMGD_ERR_UNIMPLEMENTED;
@@ -346,7 +346,7 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     // a chain that spans clusters keeps only its slice of the peers' packets in shared memory: more room for rows
     const bool multi = L.cpc > 1;
     fixed_smem = bmgdk::glm_smem_plan(warps, gpw, pre, 1, 0, pcap, eb, S, multi, gathered).total_bytes;
-    ring_budget = std::min(h->smem_optin - fixed_smem, 160 * 1024);
+    ring_budget = h->smem_optin - fixed_smem - 1024;  // all of the CTA's shared memory but a small reserve
     const int G = L.cpc * S;
     const int rows_per_cta = (n + G - 1) / G;
     const int subpasses = std::max(1, (rows_per_cta + spp - 1) / spp);
@@ -1053,6 +1053,12 @@ int bmgd_last_cuda_error(const bmgd_t* h) { return h ? h->last_cuda : 0; }
 int bmgd_debug_trace(long long* out_host, int count) {
     if (!out_host || count <= 0 || count > bmgdk::kTraceSteps * bmgdk::kTracePhases) return BMGD_ERR_ARG;
     cudaError_t e = cudaMemcpyFromSymbol(out_host, bmgdk::g_trace, sizeof(long long) * (size_t)count);
+    return e == cudaSuccess ? BMGD_OK : BMGD_ERR_CUDA;
+}
+// The same for the stamps of the first producer warp (indexed by the pair of ring stages it works on).
+int bmgd_debug_producer_trace(long long* out_host, int count) {
+    if (!out_host || count <= 0 || count > bmgdk::kTraceSteps * bmgdk::kTracePhases) return BMGD_ERR_ARG;
+    cudaError_t e = cudaMemcpyFromSymbol(out_host, bmgdk::g_ptrace, sizeof(long long) * (size_t)count);
     return e == cudaSuccess ? BMGD_OK : BMGD_ERR_CUDA;
 }
 #endif

@@ -263,8 +263,16 @@ __device__ long long g_trace[kTraceSteps * kTracePhases];
         if (blockIdx.x == BMGD_TRACE_BLOCK && threadIdx.x == 0 && step_count < (uint32_t)kTraceSteps) \
             g_trace[step_count * kTracePhases + (ph)] = clock64();                                  \
     } while (0)
+// the same for the first producer warp, indexed by the pair of stages it works on
+__device__ long long g_ptrace[kTraceSteps * kTracePhases];
+#define BMGD_PSTAMP(ph)                                                                                  \
+    do {                                                                                                 \
+        if (blockIdx.x == BMGD_TRACE_BLOCK && pw == 0 && lane == 0 && (it >> 1) < (uint32_t)kTraceSteps)  \
+            g_ptrace[(it >> 1) * kTracePhases + (ph)] = clock64();                                       \
+    } while (0)
 #else
 #define BMGD_STAMP(ph) do { } while (0)
+#define BMGD_PSTAMP(ph) do { } while (0)
 #endif
 
 // ---------------------------------------------------------------- the kernel
@@ -636,6 +644,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
         uint32_t rot = (uint32_t)pw;  // (pw - pair * nbatch) mod NPW, kept incrementally: ownership of batches rotates
         const uint32_t rot_step = (uint32_t)(nbatch % NPW);
         for (uint32_t it = 0; it < total_stages; it += 2) {
+            BMGD_PSTAMP(0);
             const Cursor A = cur;
             advance(cur);
             const bool two = it + 1 < total_stages;
@@ -670,6 +679,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                 }
             }
             const uint32_t fullA = full_bars + (uint32_t)(slotA * 8), fullB = full_bars + (uint32_t)(slotB * 8);
+            BMGD_PSTAMP(1);
             bounded_mbar_wait(empty_bars + (uint32_t)(slotA * 8), parA, aborted, P);
             __syncwarp();
             uint32_t sent = 0;
@@ -678,7 +688,9 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                 const int bb = b0 + kk * NPW;
                 if (bb < nbatch) sent += copy_batch(baseA, fullA, 32 * bb, rowsA[kk]);
             }
+            BMGD_PSTAMP(3);
             finish_stage(fullA, sent);  // a producer without a batch in this stage still counts on its barrier
+            BMGD_PSTAMP(4);
             if (two) {
                 bounded_mbar_wait(empty_bars + (uint32_t)(slotB * 8), parB, aborted, P);
                 __syncwarp();
@@ -689,6 +701,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                     if (bb < nbatch) sent += copy_batch(baseB, fullB, 32 * bb, rowsB[kk]);
                 }
                 finish_stage(fullB, sent);
+                BMGD_PSTAMP(6);
             }
         }
         cp_async_wait_all();
