@@ -52,6 +52,7 @@ def parse_args():
     ap.add_argument("--threads", type=int, default=0)
     ap.add_argument("--depth", type=int, default=0)
     ap.add_argument("--subpasses", type=int, default=0, help="sub-passes per ring stage")
+    ap.add_argument("--lanes-per-row", type=int, default=0, help="lanes that share a row in the inner loop (0: library default)")
     ap.add_argument("--producer-warps", type=int, default=0, help="warps per CTA that only fetch rows (0: library default)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
@@ -268,7 +269,7 @@ def run_ours(args, w):
     host = [inputs.make_buffer(w, k) for k in range(nb)]
     seed0 = w.seed + rank * 1_000_003
     shape = dict(cluster_size=args.cluster_size, ctas_per_chain=args.ctas_per_chain, threads_per_cta=args.threads,
-                 pipeline_depth=args.depth, subpasses_per_stage=args.subpasses, producer_warps=args.producer_warps)
+                 pipeline_depth=args.depth, subpasses_per_stage=args.subpasses, producer_warps=args.producer_warps, lanes_per_row=args.lanes_per_row)
     sg_per_step = [x.shape[0] * w.T * w.Rc for x, _ in host]
 
     # ---- device-resident measurement

@@ -89,7 +89,9 @@ typedef struct bmgd_config {
     int32_t pipeline_depth;   /* row-prefetch stages held in shared memory: 2 to 8 */
     int32_t subpasses_per_stage; /* a stage holds this many sweeps of the CTA over its rows: 1, 2, 4, ... 32 */
     int32_t producer_warps;   /* linear/logistic: extra warps per CTA that only evaluate the shuffle and fetch rows: 1 to 8 */
-    int32_t reserved[6];      /* must be zero */
+    int32_t lanes_per_row;    /* linear/logistic: lanes that share one row in the inner loop: 4, 8, 16 or 32, if the row size has
+                                 a kernel built that way */
+    int32_t reserved[5];      /* must be zero */
 } bmgd_config;
 
 typedef struct bmgd_stats {

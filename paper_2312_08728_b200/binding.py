@@ -48,7 +48,7 @@ class BmgdConfig(ctypes.Structure):
         ("cluster_size", ctypes.c_int32), ("ctas_per_chain", ctypes.c_int32),
         ("threads_per_cta", ctypes.c_int32), ("pipeline_depth", ctypes.c_int32),
         ("subpasses_per_stage", ctypes.c_int32), ("producer_warps", ctypes.c_int32),
-        ("reserved", ctypes.c_int32 * 6),
+        ("lanes_per_row", ctypes.c_int32), ("reserved", ctypes.c_int32 * 5),
     ]
 
 
@@ -195,7 +195,7 @@ class Bmgd:
     def __init__(self, N: int, p: int, K: int, loss: int = LOSS_LINEAR, dtype: int = DTYPE_F32, C: int = 1,
                  Rc: int = 1, device: int = 0, flags: int = 0, cluster_size: int = 0, ctas_per_chain: int = 0,
                  threads_per_cta: int = 0, pipeline_depth: int = 0, subpasses_per_stage: int = 0,
-                 producer_warps: int = 0,
+                 producer_warps: int = 0, lanes_per_row: int = 0,
                  timeout_ms: float = 0.0,
                  use_torch_stream: bool = False):
         if not torch.cuda.is_available():
@@ -210,6 +210,7 @@ class Bmgd:
         cfg.threads_per_cta, cfg.pipeline_depth, cfg.timeout_ms = threads_per_cta, pipeline_depth, timeout_ms
         cfg.subpasses_per_stage = subpasses_per_stage
         cfg.producer_warps = producer_warps
+        cfg.lanes_per_row = lanes_per_row
         need = ctypes.c_int64()
         self._check(self._lib.bmgd_workspace_bytes(ctypes.byref(cfg), ctypes.byref(need)), "bmgd_workspace_bytes")
         self.device = torch.device("cuda", device)

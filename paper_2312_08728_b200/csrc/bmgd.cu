@@ -117,8 +117,11 @@ int validate(const bmgd_config* c) {
     }
     const int64_t N0 = (c->N + c->K - 1) / c->K;
     if (N0 > 0x7FFFFFFFll) return BMGD_ERR_ARG;
-    for (int i = 0; i < 6; ++i)
+    for (int i = 0; i < 5; ++i)
         if (c->reserved[i] != 0) return BMGD_ERR_ARG;
+    if (c->lanes_per_row != 0 && c->lanes_per_row != 4 && c->lanes_per_row != 8 && c->lanes_per_row != 16 &&
+        c->lanes_per_row != 32)
+        return BMGD_ERR_ARG;
     if (c->producer_warps < 0 || c->producer_warps > 8) return BMGD_ERR_ARG;
     if (c->cluster_size != 0 && c->cluster_size != 1 && c->cluster_size != 2 && c->cluster_size != 4 &&
         c->cluster_size != 8 && c->cluster_size != 16)
@@ -219,21 +222,26 @@ const GlmVariant* glm_variants(bool aligned16, int* count) {
                                      ? bmgdk::glm_kernel<T, VEC, LPR, KCH, LG, bmgdk::glm_max_threads<T, VEC, KCH>()> : nullptr, \
                                  VEC, LPR, KCH, \
                                  bmgdk::glm_max_consumer_threads<T, VEC, KCH>(), bmgdk::glm_max_threads<T, VEC, KCH>()}
-    static const GlmVariant wide[] = {BMGD_VAR(V, 8, 1), BMGD_VAR(V, 8, 2), BMGD_VAR(V, 8, 4),
-                                      BMGD_VAR(V, 8, 8), BMGD_VAR(V, 16, 8), BMGD_VAR(V, 32, 8)};
+    // ordered by capacity; among equal capacities the one listed first is the default, the others are reached
+    // through cfg.lanes_per_row
+    static const GlmVariant wide[] = {BMGD_VAR(V, 8, 1), BMGD_VAR(V, 8, 2), BMGD_VAR(V, 4, 4), BMGD_VAR(V, 4, 7),
+                                      BMGD_VAR(V, 8, 4), BMGD_VAR(V, 8, 8), BMGD_VAR(V, 16, 8), BMGD_VAR(V, 32, 8)};
     static const GlmVariant narrow[] = {BMGD_VAR(1, 32, 1), BMGD_VAR(1, 32, 2), BMGD_VAR(1, 32, 4), BMGD_VAR(1, 32, 8)};
 #undef BMGD_VAR
-    if (aligned16) { *count = 6; return wide; }
+    if (aligned16) { *count = 8; return wide; }
     *count = 4;
     return narrow;
 }
 
-const GlmVariant* pick_variant(int dtype, int loss, int p, bool aligned16) {
+const GlmVariant* pick_variant(int dtype, int loss, int p, bool aligned16, int lanes_per_row = 0) {
     int cnt = 0;
     const bool lg = loss == BMGD_LOSS_LOGISTIC;
     const GlmVariant* v = dtype == BMGD_F64
         ? (lg ? glm_variants<double, true>(aligned16, &cnt) : glm_variants<double, false>(aligned16, &cnt))
         : (lg ? glm_variants<float, true>(aligned16, &cnt) : glm_variants<float, false>(aligned16, &cnt));
+    if (lanes_per_row)  // the smallest variant with that many lanes per row, if there is one
+        for (int i = 0; i < cnt; ++i)
+            if (v[i].cap() >= p && v[i].lpr == lanes_per_row) return &v[i];
     for (int i = 0; i < cnt; ++i)
         if (v[i].cap() >= p) return &v[i];
     return nullptr;
@@ -282,7 +290,7 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     if (L.pwarps < 1) return BMGD_ERR_ARG;
     const int warps = L.threads / 32;
     const int spp = warps * gpw;  // rows a CTA works on at once (one sub-pass)
-    const bool pre = var->kch * var->vec <= 16;
+    const bool pre = bmgdk::glm_prereduce(var->kch * var->vec, var->lpr);
     const bool gathered = bmgdk::glm_gathered(var->vec * eb, pcap);
 
     // Cluster size.  Measured on B200: a step costs one cluster barrier (about 0.6-0.9 us) inside one cluster, and
@@ -364,7 +372,9 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     L.rb = rb;
     L.passes = (subpasses + rb - 1) / rb;
     const int stage_bytes = stage_bytes_of(rb);
-    int depth = c.pipeline_depth ? c.pipeline_depth : 4;  // ring stages: 2 to 8
+    // ring stages: 2 to 8.  Where partial sums cross clusters through global memory, copies in flight for later steps
+    // delay the packets on the same path (measured on B200: cfg3 4.8 us per step with two stages, 5.7 with three).
+    int depth = c.pipeline_depth ? c.pipeline_depth : (L.cpc > 1 ? 2 : 4);
     while (depth > 2 && depth * stage_bytes > ring_budget) --depth;
     if (depth * stage_bytes > ring_budget) return BMGD_ERR_UNIMPLEMENTED;
     L.depth = depth;
@@ -411,7 +421,7 @@ int check_status_word(bmgd* h) {
 int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, int n, double lr, uint64_t seed) {
     const bmgd_config& c = h->cfg;
     const bool aligned16 = ((int64_t)c.p * h->tb) % 16 == 0 && ((uintptr_t)dx % 16) == 0;
-    const GlmVariant* var = pick_variant(c.dtype, c.loss, c.p, aligned16);
+    const GlmVariant* var = pick_variant(c.dtype, c.loss, c.p, aligned16, c.lanes_per_row);
     if (!var) return BMGD_ERR_UNIMPLEMENTED;
     if (((uintptr_t)dx % h->tb) != 0 || ((uintptr_t)dy % h->tb) != 0) return BMGD_ERR_ARG;
     LaunchShape L{};

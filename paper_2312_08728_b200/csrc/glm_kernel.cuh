@@ -6,10 +6,12 @@
 // replicate chains there are several teams, each taking chains team, team+nteams, ...
 //
 // Per step, in every CTA:
-//   1. rows pi(j) of this CTA's share were fetched into a shared-memory ring by dedicated producer warps
-//      (16-byte cp.async chunks, completion counted on one mbarrier per ring stage), several stages ahead: rows
-//      do not depend on theta and the shuffle is stateless, so the producers run through step, round and chain
-//      boundaries and the evaluation of pi never sits on the path from one theta to the next;
+//   1. rows pi(j) of this CTA's share were fetched into a shared-memory ring by dedicated producer warps, several
+//      stages ahead: four rows per tensor-map gather (cp.async.bulk.tensor tile::gather4) where rows are 16-byte
+//      multiples of at most 256 values, one bulk copy per row where they are wider, element-wise cp.async otherwise;
+//      completion is counted on one mbarrier per ring stage.  Rows do not depend on theta and the shuffle is
+//      stateless, so the producers run through step, round and chain boundaries and the evaluation of pi never sits
+//      on the path from one theta to the next;
 //   2. in the consumer warps a group of LPR lanes owns one row: x.theta by an LPR-lane butterfly, the residual
 //      (x.theta - y, or sigmoid(x.theta) - y), then g += r * x with x still in registers, so a
 //      row is read from HBM once and from shared memory once;
@@ -281,7 +283,7 @@ __device__ long long g_ptrace[kTraceSteps * kTracePhases];
 // per-lane state (or fp64) needs a large register budget per thread.
 template <typename T, int VEC, int KCH>
 __host__ __device__ constexpr int glm_max_consumer_threads() {
-    return (sizeof(T) == 8 || KCH * VEC >= 32) ? 256 : 512;
+    return (sizeof(T) == 8 || KCH * VEC >= 24) ? 256 : 512;
 }
 // CTA sizes a kernel is compiled for (consumers plus producers; registers come in units of four warps): kGlmSmallCta
 // leaves 168 registers per thread, kGlmLargeCta 96 and is built only for variants with little per-lane state.  (A
@@ -289,12 +291,12 @@ __host__ __device__ constexpr int glm_max_consumer_threads() {
 constexpr int kGlmSmallCta = 256 + 128, kGlmLargeCta = 512 + 128;
 template <typename T, int VEC, int KCH>
 __host__ __device__ constexpr int glm_max_threads() {
-    return (sizeof(T) == 8 || KCH * VEC >= 32) ? kGlmSmallCta : kGlmLargeCta;
+    return (sizeof(T) == 8 || KCH * VEC >= 24) ? kGlmSmallCta : kGlmLargeCta;
 }
-// Few values per lane: fold the row groups of a warp together by shuffles before shared memory.
-template <int VEC, int KCH>
-__host__ __device__ constexpr bool glm_prereduce() {
-    return KCH * VEC <= 16;
+// Fold the row groups of a warp together by shuffles before shared memory where that is cheap: few values per lane,
+// or only two groups per warp (one shuffle level).  Fewer partial rows also leave more shared memory for the ring.
+__host__ __device__ constexpr bool glm_prereduce(int values_per_lane, int lanes_per_row) {
+    return values_per_lane <= 16 || (lanes_per_row >= 16 && values_per_lane <= 32);
 }
 
 // How mini-batch rows [lo, lo+nm) are dealt to CTA g of G: a contiguous run of `cnt` rows from lo+a.
@@ -482,7 +484,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
     constexpr int FPT = (PCAP + 255) / 256;  // features per thread in the reductions (at least 256 consumer threads)
     constexpr int CB = VEC * (int)sizeof(T); // copy chunk bytes
     constexpr int NW = Words<T>::N;
-    constexpr bool PRE = glm_prereduce<VEC, KCH>();
+    constexpr bool PRE = glm_prereduce(KCH * VEC, LPR);
     constexpr bool G4 = glm_gathered(CB, PCAP);  // rows arrive four at a time through the tensor map `xmap` of X
     constexpr int YOFF = PCAP * (int)sizeof(T);  // other layouts: y sits behind the predictors of its row
     constexpr uint32_t kNoRow = 0xFFFFFFFFu;

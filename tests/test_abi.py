@@ -72,7 +72,7 @@ def test_workspace_size_counts_slots_theta_and_exchange():
     (dict(K=2000), binding.ERR_ARG), (dict(loss=3), binding.ERR_ARG), (dict(dtype=7), binding.ERR_ARG),
     (dict(Rc=0), binding.ERR_ARG), (dict(C=3), binding.ERR_ARG), (dict(cluster_size=3), binding.ERR_ARG),
     (dict(threads_per_cta=100), binding.ERR_ARG), (dict(threads_per_cta=300), binding.ERR_ARG),
-    (dict(producer_warps=9), binding.ERR_ARG),
+    (dict(producer_warps=9), binding.ERR_ARG), (dict(lanes_per_row=5), binding.ERR_ARG),
     (dict(pipeline_depth=1), binding.ERR_ARG), (dict(pipeline_depth=9), binding.ERR_ARG),
     (dict(loss=2, C=1, dtype=2), binding.ERR_ARG), (dict(loss=2, C=10, dtype=1), binding.ERR_UNIMPLEMENTED),
     (dict(loss=0, dtype=2), binding.ERR_UNIMPLEMENTED), (dict(N=2**40, K=1), binding.ERR_ARG),

@@ -122,6 +122,17 @@ def test_predictor_counts_including_unaligned_rows(dtype, p):
     check(w, buffers_of(w), mode="resident")
 
 
+@pytest.mark.parametrize("dtype,p,lanes", [(DTYPE_F32, 40, 4), (DTYPE_F32, 64, 4), (DTYPE_F32, 64, 8), (DTYPE_F32, 100, 4),
+                                           (DTYPE_F32, 100, 8), (DTYPE_F32, 112, 0), (DTYPE_F64, 20, 4), (DTYPE_F64, 56, 4),
+                                           (DTYPE_F64, 56, 8), (DTYPE_F32, 300, 4)])
+def test_lanes_per_row_variants(dtype, p, lanes):
+    """Row sizes that have kernels with four and with eight lanes per row give the same theta either way (a row size
+    without the asked-for kernel falls back to the default one); chains and a ragged last mini-batch included."""
+    w = Workload("lanes", LOSS_LOGISTIC, dtype, N=3_100, p=p, K=1, n=500, T=2, lr=0.3, epochs=1, Rc=3, seed=100 + p)
+    check(w, buffers_of(w), mode="resident", lanes_per_row=lanes)
+    check(w, buffers_of(w), mode="resident", lanes_per_row=lanes, cluster_size=4, ctas_per_chain=8)
+
+
 @pytest.mark.parametrize("N0,n", [(1, 1), (7, 1), (7, 7), (7, 100), (33, 32), (1000, 999), (1000, 1000), (257, 3)])
 def test_degenerate_sizes(N0, n):
     """One row, one-row mini-batches, a full-batch round, a batch larger than the buffer, a one-row tail."""
