@@ -301,9 +301,10 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     if (S == 0) {
         if (c.Rc > 1) S = std::min(8, floor_pow2(std::max(1, h->sm_count / c.Rc)));
         else S = 16;
-        // do not spread a mini-batch thinner than one sweep of a CTA over its rows: below that a larger cluster only
-        // adds exchange latency (measured on B200: n = 100 runs fastest on 2 CTAs)
-        while (S > 1 && n / S < spp) S /= 2;
+        // do not spread a mini-batch thinner than two sweeps of a CTA over its rows: below that a larger cluster only
+        // adds exchange latency (measured on B200, n = 100 in fp64: 1.46 us per step on one CTA, 1.58-1.71 on two, 1.65 on
+        // four, 1.9 on eight)
+        while (S > 1 && n / S < 2 * spp) S /= 2;
     }
 
     // How many clusters can be resident depends on shared memory, which depends on the ring; ask with
