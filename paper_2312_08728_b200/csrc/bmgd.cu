@@ -279,8 +279,9 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     const int pcap = var->cap();
     LaunchShape L{};
     // Replicate chains keep every SM busy with several chains' rows in flight: throughput, not the per-step latency,
-    // sets the pace there, so the CTA is as large as the register file allows (measured on B200: 16 consumer warps
-    // and 4 producer warps beat 12 + 8 and 14 + 6 once rows arrive four per gather).
+    // sets the pace there, so variants with little per-lane state run as large a CTA as the register file allows
+    // (measured on B200: 16 consumer warps and 4 producer warps beat 12 + 8 and 14 + 6 once rows arrive four per
+    // gather).  Variants with wide per-lane state always run 8 consumer warps at 168 registers.
     const bool throughput = c.Rc > 1 && var->max_consumer_threads() >= 512;
     L.threads = c.threads_per_cta ? std::min(c.threads_per_cta, var->max_consumer_threads()) : (throughput ? 512 : 256);
     // Producer warps only evaluate the shuffle and issue copies; both are chains of dependent instructions, so several
@@ -293,9 +294,9 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     const bool pre = bmgdk::glm_prereduce(var->kch * var->vec, var->lpr);
     const bool gathered = bmgdk::glm_gathered(var->vec * eb, pcap);
 
-    // Cluster size.  Measured on B200: a step costs one cluster barrier (about 0.6-0.9 us) inside one cluster, and
-    // about 2.5 us more once partial sums have to cross clusters through L2, while a sub-pass of spp rows costs about
-    // 0.35 us.  So a chain gets the largest cluster the device admits and stays inside it unless a CTA would have to
+    // Cluster size.  Measured on B200: a step costs one exchange through distributed shared memory (about 0.8 us among
+    // 16 CTAs) inside one cluster, and about 2.5 us more once partial sums have to cross clusters through L2, while a
+    // sub-pass of spp rows costs about 0.15-0.3 us.  So a chain gets the largest cluster the device admits and stays inside it unless a CTA would have to
     // sweep many sub-passes per step.
     int S = c.cluster_size;
     if (S == 0) {
@@ -628,9 +629,8 @@ int bmgd_create_ex(const bmgd_config* cfg, bmgd_t** out) {
     h->lay = make_layout(cfg);
 
     auto fail = [&](int code) { bmgd_destroy(h); return code; };
-    cudaError_t e;
-    if ((e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess ||
-        (e = cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess) {
+    if (cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&h->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
         cudaGetLastError();
         return fail(BMGD_ERR_CUDA);
     }

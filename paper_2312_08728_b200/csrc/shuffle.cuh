@@ -76,8 +76,9 @@ __host__ __device__ __forceinline__ RoundKeys round_keys(uint64_t seed, uint32_t
 }
 
 __host__ __device__ __forceinline__ uint32_t feistel_f(uint32_t v, uint32_t k) {
-    const uint32_t w = v + k;
-    return mulhi32(0xD2511F53u, w) ^ (0xD2511F53u * w);
+    // one 32 x 32 -> 64 bit multiply gives both halves
+    const unsigned long long pr = (unsigned long long)0xD2511F53u * (unsigned long long)(uint32_t)(v + k);
+    return (uint32_t)(pr >> 32) ^ (uint32_t)pr;
 }
 
 __host__ __device__ __forceinline__ uint32_t perm_index(uint32_t j, const FeistelDomain& d, const RoundKeys& rk) {
