@@ -91,7 +91,10 @@ typedef struct bmgd_config {
     int32_t producer_warps;   /* linear/logistic: extra warps per CTA that only evaluate the shuffle and fetch rows: 1 to 8 */
     int32_t lanes_per_row;    /* linear/logistic: lanes that share one row in the inner loop: 4, 8, 16 or 32, if the row size has
                                  a kernel built that way */
-    int32_t reserved[5];      /* must be zero */
+    int32_t first_chain;      /* shuffle id of this handle's first chain: chain c of the handle draws the partitions of
+                                 chain first_chain + c, so the chains of one job can be spread over several handles (one
+                                 per GPU) and give, bit for bit, what one handle with all of them gives; default 0 */
+    int32_t reserved[4];      /* must be zero */
 } bmgd_config;
 
 typedef struct bmgd_stats {
@@ -226,6 +229,12 @@ int bmgd_set_optimizer(bmgd_t* h, int32_t kind, double a, double b, double eps);
 enum { BMGD_LR_CONSTANT = 0, BMGD_LR_COSINE = 1 };
 int bmgd_set_lr_schedule(bmgd_t* h, int32_t kind, int64_t updates_per_pass);
 
+/* Change the bound on any single device-side wait of later launches (cfg.timeout_ms at creation): a wait that
+ * lasts longer gives up, the launch ends early without writing theta back, and the next synchronising call returns
+ * BMGD_ERR_TIMEOUT once; the handle stays usable.  <= 0 selects 2000 ms.  A bound below one microsecond makes every
+ * wait that does not succeed at its first look give up (for testing the error path without hanging a GPU). */
+int bmgd_set_timeout(bmgd_t* h, double timeout_ms);
+
 /* Synchronise and fill *out. */
 int bmgd_get_stats(bmgd_t* h, bmgd_stats* out);
 
@@ -251,6 +260,16 @@ int bmgd_partition_index(uint64_t seed, uint32_t pass, int64_t N, int64_t j, int
 int bmgd_gather_buffer(const void* host_x, const void* host_y, int64_t N, int64_t row_bytes, int64_t y_bytes,
                        int32_t K, uint64_t seed, uint32_t pass, int32_t k, void* stage_x, void* stage_y,
                        int32_t threads, int64_t* rows_out);
+
+/* Latency probe of the computation step (linear and logistic handles): launch, on the compute stream, the step
+ * kernel's own synchronisation structure for a buffer of `rows` rows, `rounds` rounds and mini-batches of
+ * batch_size rows, in the launch shape bmgd_run_rounds would choose, with every ring hand-over, barrier, packet
+ * exchange between CTAs and update of a step, but without fetching or multiplying a single row (the gradient is
+ * zero, so theta, the update rule's state and the step counters stay as they are).  Timed like any launch under
+ * BMGD_FLAG_TIMING (bmgd_get_stats: launches, kernel_ms).  Its time per step is the floor that the dependency of
+ * each step on the one before (Eq. (2.1)) puts under the step time of a single chain, whatever the memory system
+ * delivers. */
+int bmgd_debug_null_rounds(bmgd_t* h, int64_t rows, int32_t rounds, int32_t batch_size);
 
 /* Launch, on the compute stream, a one-thread kernel that waits with the step kernels' bounded-wait protocol for
  * something that never happens, with a budget of budget_ms (at most 1000).  The wait gives up, the kernel returns,

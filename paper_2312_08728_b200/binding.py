@@ -32,7 +32,7 @@ EXPORTS = (
     "bmgd_load_buffer", "bmgd_run_rounds", "bmgd_run_rounds_resident", "bmgd_sync", "bmgd_get_theta",
     "bmgd_set_theta", "bmgd_get_stats", "bmgd_debug_perm", "bmgd_strerror", "bmgd_last_cuda_error",
     "bmgd_version", "bmgd_run_rounds_noalloc", "bmgd_debug_wait_timeout", "bmgd_partition_index", "bmgd_gather_buffer",
-    "bmgd_set_optimizer", "bmgd_set_lr_schedule",
+    "bmgd_set_optimizer", "bmgd_set_lr_schedule", "bmgd_set_timeout", "bmgd_debug_null_rounds",
 )
 
 OPT_SGD, OPT_NESTEROV, OPT_ADAM = 0, 1, 2
@@ -48,7 +48,7 @@ class BmgdConfig(ctypes.Structure):
         ("cluster_size", ctypes.c_int32), ("ctas_per_chain", ctypes.c_int32),
         ("threads_per_cta", ctypes.c_int32), ("pipeline_depth", ctypes.c_int32),
         ("subpasses_per_stage", ctypes.c_int32), ("producer_warps", ctypes.c_int32),
-        ("lanes_per_row", ctypes.c_int32), ("reserved", ctypes.c_int32 * 5),
+        ("lanes_per_row", ctypes.c_int32), ("first_chain", ctypes.c_int32), ("reserved", ctypes.c_int32 * 4),
     ]
 
 
@@ -103,6 +103,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.bmgd_sync.argtypes = [vp]
     L.bmgd_set_optimizer.argtypes = [vp, i32, dbl, dbl, dbl]
     L.bmgd_set_lr_schedule.argtypes = [vp, i32, i64]
+    L.bmgd_set_timeout.argtypes = [vp, dbl]
     L.bmgd_get_theta.argtypes = [vp, vp, i64]
     L.bmgd_set_theta.argtypes = [vp, vp, i64]
     L.bmgd_get_stats.argtypes = [vp, P(BmgdStats)]
@@ -111,6 +112,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.bmgd_last_cuda_error.argtypes = [vp]
     L.bmgd_version.argtypes = []
     L.bmgd_debug_wait_timeout.argtypes = [vp, dbl]
+    L.bmgd_debug_null_rounds.argtypes = [vp, i64, i32, i32]
     L.bmgd_partition_index.argtypes = [u64, u32, i64, i64, P(i64)]
     L.bmgd_gather_buffer.argtypes = [vp, vp, i64, i64, i64, i32, u64, u32, i32, vp, vp, i32, P(i64)]
     L.bmgd_run_rounds_noalloc.argtypes = [vp, vp, i64, i32, i32, i32, i32, vp, i32, i32, dbl, u64, vp]
@@ -128,6 +130,37 @@ _NP_THETA = {DTYPE_F64: np.float64, DTYPE_F32: np.float32, DTYPE_BF16: np.float3
 
 NOALLOC_MAX_P = 256
 
+_TORCH_X = {DTYPE_F64: torch.float64, DTYPE_F32: torch.float32, DTYPE_BF16: torch.bfloat16}
+_TORCH_THETA = {DTYPE_F64: torch.float64, DTYPE_F32: torch.float32, DTYPE_BF16: torch.float32}
+
+
+def check_buffer(x: torch.Tensor, y: torch.Tensor, p: int, loss: int, dtype: int, max_rows: Optional[int] = None) -> int:
+    """Refuse a buffer whose tensors do not have the shape and element types the job was created for.
+
+    The C ABI takes bare pointers, so a float32 X handed to a float64 job, an X with another column count, a
+    shorter y or labels that are not int32 would make the kernel read past the end of an allocation.  This is
+    the only place where the tensors' own metadata can be compared with the job.  Returns the row count."""
+    if dtype not in _TORCH_X:
+        raise ValueError(f"unknown dtype code {dtype}")
+    if x.dim() != 2 or x.shape[1] != p:
+        raise ValueError(f"X must be [rows, {p}], got {tuple(x.shape)}")
+    if x.dtype != _TORCH_X[dtype]:
+        raise ValueError(f"X must be {_TORCH_X[dtype]}, got {x.dtype}")
+    want_y = torch.int32 if loss == LOSS_SOFTMAX else _TORCH_THETA[dtype]
+    if y.dim() != 1 or y.shape[0] != x.shape[0]:
+        raise ValueError(f"y must be [{x.shape[0]}], got {tuple(y.shape)}")
+    if y.dtype != want_y:
+        raise ValueError(f"y must be {want_y}, got {y.dtype}")
+    if not (x.is_contiguous() and y.is_contiguous()):
+        raise ValueError("X and y must be contiguous")
+    if x.device != y.device:
+        raise ValueError("X and y must live on the same device")
+    if x.shape[0] < 1:
+        raise ValueError("a buffer needs at least one row")
+    if max_rows is not None and x.shape[0] > max_rows:
+        raise ValueError(f"{x.shape[0]} rows do not fit a slot of {max_rows}")
+    return x.shape[0]
+
 
 def run_rounds_noalloc(dev_x: torch.Tensor, dev_y: torch.Tensor, theta: torch.Tensor, loss: int, dtype: int,
                        rounds: int, batch_size: int, lr: float, seed: int,
@@ -140,10 +173,19 @@ def run_rounds_noalloc(dev_x: torch.Tensor, dev_y: torch.Tensor, theta: torch.Te
     passed as they are and must already be contiguous and on the current device.  Returns once the
     kernel has finished; calls on one GPU must not overlap, they share one fixed scratch array.
     """
+    if theta.dim() != 2:
+        raise ValueError(f"theta must be [Rc, p], got {tuple(theta.shape)}")
+    Rc, p = theta.shape
+    # y is checked as a response vector in the parameter type: the entry point has no softmax kernel, and the
+    # library itself refuses such a job
+    check_buffer(dev_x, dev_y, p, LOSS_LINEAR, dtype)
+    if theta.dtype != _TORCH_THETA[dtype]:
+        raise ValueError(f"theta must be {_TORCH_THETA[dtype]}, got {theta.dtype}")
     for t in (dev_x, dev_y, theta):
         if t.device.type != "cuda" or not t.is_contiguous():
             raise ValueError("run_rounds_noalloc takes contiguous device tensors")
-    Rc, p = theta.shape
+    if theta.device != dev_x.device:
+        raise ValueError("theta and the buffer must live on the same device")
     L = load_library()
     s = stream.cuda_stream if stream is not None else None
     rc = L.bmgd_run_rounds_noalloc(dev_x.data_ptr(), dev_y.data_ptr(), dev_x.shape[0], p, loss, dtype, Rc,
@@ -196,7 +238,7 @@ class Bmgd:
                  Rc: int = 1, device: int = 0, flags: int = 0, cluster_size: int = 0, ctas_per_chain: int = 0,
                  threads_per_cta: int = 0, pipeline_depth: int = 0, subpasses_per_stage: int = 0,
                  producer_warps: int = 0, lanes_per_row: int = 0,
-                 timeout_ms: float = 0.0,
+                 timeout_ms: float = 0.0, first_chain: int = 0,
                  use_torch_stream: bool = False):
         if not torch.cuda.is_available():
             raise RuntimeError("BMGD needs a CUDA device; there is no CPU path")
@@ -211,6 +253,7 @@ class Bmgd:
         cfg.subpasses_per_stage = subpasses_per_stage
         cfg.producer_warps = producer_warps
         cfg.lanes_per_row = lanes_per_row
+        cfg.first_chain = first_chain
         need = ctypes.c_int64()
         self._check(self._lib.bmgd_workspace_bytes(ctypes.byref(cfg), ctypes.byref(need)), "bmgd_workspace_bytes")
         self.device = torch.device("cuda", device)
@@ -242,9 +285,9 @@ class Bmgd:
         """Start the host-to-device copy of one buffer; returns the slot id."""
         if host_x.device.type != "cpu" or host_y.device.type != "cpu":
             raise ValueError("load_buffer takes host tensors")
-        if not (host_x.is_contiguous() and host_y.is_contiguous()):
-            raise ValueError("host buffers must be contiguous")
-        rows = host_x.shape[0]
+        rows = check_buffer(host_x, host_y, self.p, self.loss, self.dtype)
+        if rows > -(-self.N // self.K):  # the library refuses it too; said here with the same status
+            raise BmgdError(ERR_CAPACITY, "load_buffer")
         slot = ctypes.c_int32(-1)
         s = stream.cuda_stream if stream is not None else None
         self._check(self._lib.bmgd_load_buffer(self._h, host_x.data_ptr(), host_y.data_ptr(), rows, s,
@@ -262,8 +305,7 @@ class Bmgd:
                             lr: float, seed: int) -> None:
         if dev_x.device != self.device or dev_y.device != self.device:
             raise ValueError("resident buffers must live on the handle's device")
-        if not (dev_x.is_contiguous() and dev_y.is_contiguous()):
-            raise ValueError("resident buffers must be contiguous")
+        check_buffer(dev_x, dev_y, self.p, self.loss, self.dtype)
         self._check(self._lib.bmgd_run_rounds_resident(self._h, dev_x.data_ptr(), dev_y.data_ptr(), dev_x.shape[0],
                                                        rounds, batch_size, float(lr),
                                                        int(seed) & 0xFFFFFFFFFFFFFFFF), "bmgd_run_rounds_resident")
@@ -291,6 +333,10 @@ class Bmgd:
         """LR_CONSTANT, or LR_COSINE: the j-th update of a pass of `updates_per_pass` takes lr (1/2 + 1/2 cos(j pi / J))."""
         self._check(self._lib.bmgd_set_lr_schedule(self._h, kind, int(updates_per_pass)), "bmgd_set_lr_schedule")
 
+    def set_timeout(self, timeout_ms: float) -> None:
+        """Bound on any single device-side wait of later launches; <= 0 selects the default of 2000 ms."""
+        self._check(self._lib.bmgd_set_timeout(self._h, float(timeout_ms)), "bmgd_set_timeout")
+
     def get_stats(self) -> dict:
         st = BmgdStats()
         self._check(self._lib.bmgd_get_stats(self._h, ctypes.byref(st)), "bmgd_get_stats")
@@ -304,6 +350,10 @@ class Bmgd:
 
     def debug_wait_timeout(self, budget_ms: float) -> None:
         self._check(self._lib.bmgd_debug_wait_timeout(self._h, float(budget_ms)), "bmgd_debug_wait_timeout")
+
+    def debug_null_rounds(self, rows: int, rounds: int, batch_size: int) -> None:
+        """Launch the step kernel's latency probe: all waits, exchanges and updates of `rounds` rounds, no rows."""
+        self._check(self._lib.bmgd_debug_null_rounds(self._h, rows, rounds, batch_size), "bmgd_debug_null_rounds")
 
     def close(self) -> None:
         if getattr(self, "_h", None) is not None and self._h:

@@ -117,8 +117,10 @@ int validate(const bmgd_config* c) {
     }
     const int64_t N0 = (c->N + c->K - 1) / c->K;
     if (N0 > 0x7FFFFFFFll) return BMGD_ERR_ARG;
-    for (int i = 0; i < 5; ++i)
+    for (int i = 0; i < 4; ++i)
         if (c->reserved[i] != 0) return BMGD_ERR_ARG;
+    if (c->first_chain < 0 || (int64_t)c->first_chain + c->Rc > 0x7FFFFFFFll) return BMGD_ERR_ARG;
+    if (c->first_chain != 0 && c->loss == BMGD_LOSS_SOFTMAX) return BMGD_ERR_UNIMPLEMENTED;
     if (c->lanes_per_row != 0 && c->lanes_per_row != 4 && c->lanes_per_row != 8 && c->lanes_per_row != 16 &&
         c->lanes_per_row != 32)
         return BMGD_ERR_ARG;
@@ -207,12 +209,23 @@ typedef void (*GlmKernel)(const GlmParams, const CUtensorMap);
 struct GlmVariant {
     GlmKernel fn_small;  // compiled for CTAs of up to kGlmSmallCta threads (more registers per thread)
     GlmKernel fn_large;  // compiled for CTAs of up to kGlmLargeCta threads, or null
-    GlmKernel fn(int cta_threads) const { return (cta_threads > bmgdk::kGlmSmallCta && fn_large) ? fn_large : fn_small; }
+    GlmKernel null_small, null_large;  // the latency probe of the same shape (least-squares tables only)
+    GlmKernel fn(int cta_threads, bool null_step = false) const {
+        const bool large = cta_threads > bmgdk::kGlmSmallCta && fn_large;
+        return null_step ? (large ? null_large : null_small) : (large ? fn_large : fn_small);
+    }
     int vec, lpr, kch, maxc, maxt;
     int cap() const { return vec * lpr * kch; }
     int max_consumer_threads() const { return maxc; }  // warps that compute
     int max_threads() const { return maxt; }           // consumers plus producers
 };
+
+// The latency probe does not depend on the loss: it is built once, beside the least-squares kernels.
+template <typename T, int VEC, int LPR, int KCH, bool LG, int MAXT>
+constexpr GlmKernel glm_null_kernel() {
+    if constexpr (LG) return nullptr;
+    else return bmgdk::glm_kernel<T, VEC, LPR, KCH, false, MAXT, true>;
+}
 
 template <typename T, bool LG>
 const GlmVariant* glm_variants(bool aligned16, int* count) {
@@ -220,6 +233,9 @@ const GlmVariant* glm_variants(bool aligned16, int* count) {
 #define BMGD_VAR(VEC, LPR, KCH) {bmgdk::glm_kernel<T, VEC, LPR, KCH, LG, bmgdk::kGlmSmallCta>, \
                                  (bmgdk::glm_max_threads<T, VEC, KCH>() != bmgdk::kGlmSmallCta) \
                                      ? bmgdk::glm_kernel<T, VEC, LPR, KCH, LG, bmgdk::glm_max_threads<T, VEC, KCH>()> : nullptr, \
+                                 glm_null_kernel<T, VEC, LPR, KCH, LG, bmgdk::kGlmSmallCta>(), \
+                                 (bmgdk::glm_max_threads<T, VEC, KCH>() != bmgdk::kGlmSmallCta) \
+                                     ? glm_null_kernel<T, VEC, LPR, KCH, LG, bmgdk::glm_max_threads<T, VEC, KCH>()>() : nullptr, \
                                  VEC, LPR, KCH, \
                                  bmgdk::glm_max_consumer_threads<T, VEC, KCH>(), bmgdk::glm_max_threads<T, VEC, KCH>()}
     // ordered by capacity; among equal capacities the one listed first is the default, the others are reached
@@ -247,6 +263,14 @@ const GlmVariant* pick_variant(int dtype, int loss, int p, bool aligned16, int l
     return nullptr;
 }
 
+// How often a waiting thread looks at the clock and the abort flag.  A budget below a microsecond cannot be measured
+// by counting polls: then every failed poll looks, so that any wait that does not succeed at once gives up.
+void set_poll_cadence(GlmParams* P) {
+    const bool tiny = P->timeout_ns < 1000ull;
+    P->poll_mask = tiny ? 0u : 0x3FFu;
+    P->mbar_mask = tiny ? 0u : 0x3Fu;
+}
+
 int floor_pow2(int v) {
     int r = 1;
     while (r * 2 <= v) r *= 2;
@@ -272,7 +296,7 @@ int max_active_clusters(bmgd* h, GlmKernel fn, int S, int threads, int smem, int
     return BMGD_OK;
 }
 
-int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* out) {
+int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* out, bool null_step = false) {
     const bmgd_config& c = h->cfg;
     const int eb = h->tb;
     const int gpw = 32 / var->lpr;
@@ -319,11 +343,11 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
             return BMGD_ERR_UNIMPLEMENTED;
         }
         const int probe_smem = fixed_smem + ring_budget;
-        BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn(L.threads + 32 * L.pwarps), cudaFuncAttributeMaxDynamicSharedMemorySize, probe_smem));
-        BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn(L.threads + 32 * L.pwarps), cudaFuncAttributeNonPortableClusterSizeAllowed, S > 8 ? 1 : 0));
+        BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn(L.threads + 32 * L.pwarps, null_step), cudaFuncAttributeMaxDynamicSharedMemorySize, probe_smem));
+        BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn(L.threads + 32 * L.pwarps, null_step), cudaFuncAttributeNonPortableClusterSizeAllowed, S > 8 ? 1 : 0));
         max_clusters = h->sm_count;
         if (S > 1) {
-            int rc = max_active_clusters(h, var->fn(L.threads + 32 * L.pwarps), S, L.threads + 32 * L.pwarps, probe_smem, &max_clusters);
+            int rc = max_active_clusters(h, var->fn(L.threads + 32 * L.pwarps, null_step), S, L.threads + 32 * L.pwarps, probe_smem, &max_clusters);
             if (rc != BMGD_OK) {
                 if (c.cluster_size == 0 && S > 8) { S = 8; continue; }  // clusters of 16 are optional in hardware
                 return rc;
@@ -420,14 +444,17 @@ int check_status_word(bmgd* h) {
     return BMGD_OK;
 }
 
-int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, int n, double lr, uint64_t seed) {
+// null_step: launch the latency probe of the same shape instead (dx and dy are not read; theta and the update rule's
+// state stay as they are).
+int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, int n, double lr, uint64_t seed,
+            bool null_step = false) {
     const bmgd_config& c = h->cfg;
     const bool aligned16 = ((int64_t)c.p * h->tb) % 16 == 0 && ((uintptr_t)dx % 16) == 0;
-    const GlmVariant* var = pick_variant(c.dtype, c.loss, c.p, aligned16, c.lanes_per_row);
+    const GlmVariant* var = pick_variant(c.dtype, null_step ? BMGD_LOSS_LINEAR : c.loss, c.p, aligned16, c.lanes_per_row);
     if (!var) return BMGD_ERR_UNIMPLEMENTED;
     if (((uintptr_t)dx % h->tb) != 0 || ((uintptr_t)dy % h->tb) != 0) return BMGD_ERR_ARG;
     LaunchShape L{};
-    int rc = plan_glm(h, var, rows, n, &L);
+    int rc = plan_glm(h, var, rows, n, &L, null_step);
     if (rc != BMGD_OK) return rc;
 
     const uint32_t M = (uint32_t)((rows + n - 1) / n);
@@ -457,6 +484,7 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
     P.adam_b1pow0 = std::pow(h->opt_a, (double)h->opt_steps);
     P.adam_b2pow0 = std::pow(h->opt_b, (double)h->opt_steps);
     P.sched = h->sched; P.sched_period = h->sched_period; P.sched_pos0 = h->sched_pos;
+    if (null_step) { P.opt_kind = bmgdk::kOptSgd; P.sched = bmgdk::kLrConstant; }  // a zero gradient under Eq. (2.1): nothing changes
     P.N0 = (uint32_t)rows; P.n = (uint32_t)n; P.M = M; P.T = rounds; P.p = c.p;
     P.Rc = c.Rc; P.S = L.S; P.cpc = L.cpc; P.nteams = L.nteams;
     P.passes = L.passes; P.rb = L.rb; P.depth = L.depth;
@@ -464,7 +492,9 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
     P.q_full = (uint32_t)n / (uint32_t)(L.cpc * L.S); P.r_full = (uint32_t)n % (uint32_t)(L.cpc * L.S);
     P.ll_stride = c.p * 2;
     P.tag_base = (uint32_t)h->tag_base;
+    P.chain0 = (uint32_t)c.first_chain;
     P.fixed_partition = (c.flags & BMGD_FLAG_FIXED_PARTITION) ? 1 : 0;
+    set_poll_cadence(&P);
     if ((int64_t)L.nteams * L.cpc > kMaxClustersForExchange) return BMGD_ERR_LAUNCH;
 
     cudaLaunchConfig_t lc{};
@@ -495,14 +525,14 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
     }
     CUtensorMap xmap;
     std::memset(&xmap, 0, sizeof xmap);
-    if (bmgdk::glm_gathered(var->vec * h->tb, var->cap())) {
+    if (!null_step && bmgdk::glm_gathered(var->vec * h->tb, var->cap())) {
         rc = make_row_map(dx, rows, c.p, h->tb, var->cap(), &xmap);
         if (rc != BMGD_OK) {
             if (timing) h->event_pool.push_back(ep);
             return rc;
         }
     }
-    cudaError_t e = cudaLaunchKernelEx(&lc, var->fn(L.threads + 32 * L.pwarps), P, xmap);
+    cudaError_t e = cudaLaunchKernelEx(&lc, var->fn(L.threads + 32 * L.pwarps, null_step), P, xmap);
     if (e != cudaSuccess) {
         h->last_cuda = (int)e;
         cudaGetLastError();
@@ -515,11 +545,13 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
         h->kernel_events.push_back(ep);
     }
     h->tag_base += steps_per_team;
-    h->opt_steps += (int64_t)rounds * M;
-    if (h->sched == BMGD_LR_COSINE) h->sched_pos = (h->sched_pos + (int64_t)rounds * M) % h->sched_period;
     h->stats.launches += 1;
-    h->stats.steps += (int64_t)c.Rc * rounds * M;
-    h->stats.sample_grads += (int64_t)c.Rc * rounds * rows;
+    if (!null_step) {
+        h->opt_steps += (int64_t)rounds * M;
+        if (h->sched == BMGD_LR_COSINE) h->sched_pos = (h->sched_pos + (int64_t)rounds * M) % h->sched_period;
+        h->stats.steps += (int64_t)c.Rc * rounds * M;
+        h->stats.sample_grads += (int64_t)c.Rc * rounds * rows;
+    }
     h->stats.grid_ctas = L.nteams * L.cpc * L.S;
     h->stats.cluster_size = L.S;
     h->stats.ctas_per_chain = L.cpc * L.S;
@@ -794,6 +826,12 @@ int bmgd_set_optimizer(bmgd_t* h, int32_t kind, double a, double b, double eps) 
     return BMGD_OK;
 }
 
+int bmgd_set_timeout(bmgd_t* h, double timeout_ms) {
+    if (!h || !std::isfinite(timeout_ms)) return BMGD_ERR_ARG;
+    h->timeout_ns = (uint64_t)((timeout_ms > 0 ? timeout_ms : 2000.0) * 1e6);
+    return BMGD_OK;
+}
+
 int bmgd_set_lr_schedule(bmgd_t* h, int32_t kind, int64_t updates_per_pass) {
     if (!h) return BMGD_ERR_ARG;
     if (kind != BMGD_LR_CONSTANT && kind != BMGD_LR_COSINE) return BMGD_ERR_ARG;
@@ -936,6 +974,7 @@ int bmgd_run_rounds_noalloc(const void* dev_x, const void* dev_y, int64_t rows, 
     P.ll_stride = p * 2;
     P.tag_base = 0;
     P.fixed_partition = 0;
+    set_poll_cadence(&P);
 
     cudaLaunchConfig_t lc{};
     lc.gridDim = dim3((unsigned)(L.nteams * L.cpc * L.S), 1, 1);
@@ -1025,6 +1064,18 @@ int bmgd_gather_buffer(const void* host_x, const void* host_y, int64_t N, int64_
     }
     for (auto& th : pool) th.join();
     return BMGD_OK;
+}
+
+int bmgd_debug_null_rounds(bmgd_t* h, int64_t rows, int32_t rounds, int32_t batch_size) {
+    if (!h) return BMGD_ERR_ARG;
+    if (h->cfg.loss == BMGD_LOSS_SOFTMAX) return BMGD_ERR_UNIMPLEMENTED;
+    if (rows <= 0 || rows > 0x7FFFFFFFll || rounds < 0 || batch_size <= 0) return BMGD_ERR_ARG;
+    if (rounds == 0) return BMGD_OK;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return cuda_fail(h, cudaErrorInvalidDevice);
+    const int n = batch_size > rows ? (int)rows : batch_size;
+    // the probe reads no rows; the workspace base stands in for an aligned buffer address
+    return run_glm(h, h->base, h->base, rows, rounds, n, 0.0, 0, true);
 }
 
 int bmgd_debug_wait_timeout(bmgd_t* h, double budget_ms) {

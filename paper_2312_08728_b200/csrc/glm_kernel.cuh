@@ -42,6 +42,8 @@ constexpr int kMaxCpc = 20;        // clusters per chain the packet exchange is 
 constexpr int kMaxClusterSize = 16; // CTAs per cluster
 constexpr int kMaxBatchesPerProducer = 2;  // batches of 32 row slots one producer warp takes in one ring stage
 constexpr int kStatusTimeout = -5; // == BMGD_ERR_TIMEOUT
+constexpr unsigned long long kDrainNs = 1000000ull;  // at the end of a launch: how long a warp waits for its own copies in flight
+constexpr int kCtaAbortOff = 512;  // shared-memory word (in front of the ring) through which a CTA's consumers agree to stop
 constexpr int kOptSgd = 0, kOptNesterov = 1, kOptAdam = 2;  // == BMGD_OPT_*
 constexpr int kLrConstant = 0, kLrCosine = 1;               // == BMGD_LR_*
 
@@ -82,6 +84,9 @@ struct GlmParams {
     int ll_stride;        // packets per cluster slot
     uint32_t tag_base;
     int fixed_partition;
+    uint32_t chain0;      // shuffle id of this launch's first chain (chains of one job may be spread over several handles)
+    uint32_t poll_mask;   // a packet poll looks at the clock and the abort flag every poll_mask+1 failed sweeps
+    uint32_t mbar_mask;   // the same for the waits on the ring's mbarriers
 };
 
 // ---------------------------------------------------------------- small PTX wrappers
@@ -335,6 +340,18 @@ __device__ __forceinline__ void perm_index2(uint32_t& x0, const RoundKeys& k0, u
     } while (w0 || w1);
 }
 
+// The rare part of every bounded wait: look at the clock and at the launch's abort flag.  When the budget has run
+// out, or another thread has given up, record the error (first one wins), raise the flag and stop waiting.
+__device__ __forceinline__ void wait_slow_path(unsigned long long& t0, bool& aborted, const GlmParams& P) {
+    const unsigned long long now = global_ns();
+    if (t0 == 0) t0 = now;
+    if (now - t0 > P.timeout_ns || ((volatile int*)P.status)[1] != 0) {
+        atomicCAS(P.status, 0, kStatusTimeout);
+        atomicExch(P.status + 1, 1);
+        aborted = true;
+    }
+}
+
 // Reads `count` tagged packets (NW 64-bit words each: value word in the low half, step tag in the high half) through
 // `load(k, w)` until every tag equals `tag`, then returns the sum of the values in the order k = 0, 1, ....  Packets
 // are taken CH at a time: all loads of a sweep over a chunk are issued before the first tag is checked.  The wait is
@@ -367,15 +384,7 @@ __device__ __forceinline__ T gather_packets(int count, uint32_t tag, bool& abort
                 }
             }
             if (ok) break;
-            if ((++spins & 0x3FFu) == 0u) {
-                const unsigned long long now = global_ns();
-                if (t0 == 0) t0 = now;
-                if (now - t0 > P.timeout_ns || ((volatile int*)P.status)[1] != 0) {
-                    atomicCAS(P.status, 0, kStatusTimeout);
-                    atomicExch(P.status + 1, 1);
-                    aborted = true;
-                }
-            }
+            if ((++spins & P.poll_mask) == 0u) wait_slow_path(t0, aborted, P);
         }
         if (!aborted) {
 #pragma unroll
@@ -452,15 +461,7 @@ __device__ __forceinline__ void bounded_mbar_wait(uint32_t bar, uint32_t parity,
     unsigned long long t0 = 0;
     uint32_t spins = 0;
     while (!aborted && !mbar_try_wait(bar, parity)) {
-        if ((++spins & 0x3Fu) == 0u) {
-            const unsigned long long now = global_ns();
-            if (t0 == 0) t0 = now;
-            if (now - t0 > P.timeout_ns || ((volatile int*)P.status)[1] != 0) {
-                atomicCAS(P.status, 0, kStatusTimeout);
-                atomicExch(P.status + 1, 1);
-                aborted = true;
-            }
-        }
+        if ((++spins & P.mbar_mask) == 0u) wait_slow_path(t0, aborted, P);
     }
 }
 
@@ -475,7 +476,11 @@ __device__ __forceinline__ void bounded_mbar_wait(uint32_t bar, uint32_t parity,
 // row beyond p is zeroed once and never written, and a slot without a row is zero-filled by its copy, so the
 // inner loop carries no predicates.  Each stage has a "full" mbarrier (the producers' copies have landed) and an
 // "empty" one (every consumer warp has read it).
-template <typename T, int VEC, int LPR, int KCH, bool LOGISTIC, int MAXT>
+//
+// NULLSTEP = true is the latency probe of the same kernel: every wait, barrier, packet exchange and update of a step
+// runs with the same launch shape, but no row is fetched and none is multiplied (the gradient is zero and theta
+// stays as it is).  Its time per step is what the step's synchronisation structure alone costs.
+template <typename T, int VEC, int LPR, int KCH, bool LOGISTIC, int MAXT, bool NULLSTEP = false>
 __global__ void __launch_bounds__(MAXT, 1)
 glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
     constexpr int GPW = 32 / LPR;            // row groups per warp
@@ -514,6 +519,8 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
 
     // zero all of shared memory once: row tails beyond p and packet tags must read as zero
     for (int i = plan.ring_off + tid * 16; i < plan.total_bytes; i += (int)blockDim.x * 16) st_shared_zero16(smem_u32(smem + i));
+    volatile int* const cta_abort = reinterpret_cast<volatile int*>(smem + kCtaAbortOff);
+    if (tid == 0) *cta_abort = 0;
     if (tid < D) {
         // every producer lane, once its element copies have landed; with bulk row copies, also one lane per producer
         // warp announcing that warp's byte count
@@ -561,7 +568,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
         };
         Cursor cur;
         cur.ci = 0; cur.t = 0; cur.sidx = 0; cur.m = 0u;
-        cur.rk = round_keys(P.seed, (uint32_t)team, 0u);
+        cur.rk = round_keys(P.seed, P.chain0 + (uint32_t)team, 0u);
         cur.sh = row_share(0u, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full);
         auto advance = [&](Cursor& c) {
             if (++c.sidx == passes) {
@@ -570,7 +577,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                     c.m = 0;
                     if (++c.t == T_rounds) { c.t = 0; ++c.ci; }
                     if (c.ci < nch)
-                        c.rk = round_keys(P.seed, (uint32_t)(team + c.ci * P.nteams), P.fixed_partition ? 0u : (uint32_t)c.t);
+                        c.rk = round_keys(P.seed, P.chain0 + (uint32_t)(team + c.ci * P.nteams), P.fixed_partition ? 0u : (uint32_t)c.t);
                 }
                 c.sh = row_share(c.m, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full);
             }
@@ -643,6 +650,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
             }
         };
 
+        uint32_t issued_mask = 0, issued_par = 0;  // ring slots this warp has sent copies into, and the parity of the last such phase
         uint32_t rot = (uint32_t)pw;  // (pw - pair * nbatch) mod NPW, kept incrementally: ownership of batches rotates
         const uint32_t rot_step = (uint32_t)(nbatch % NPW);
         for (uint32_t it = 0; it < total_stages; it += 2) {
@@ -668,7 +676,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
             for (int kk = 0; kk < kMaxBatchesPerProducer; ++kk) {
                 const int bb = b0 + kk * NPW;
                 rowsA[kk] = kNoRow; rowsB[kk] = kNoRow;
-                if (bb < nbatch) {
+                if (!NULLSTEP && bb < nbatch) {
                     const int s = 32 * bb + lane;
                     const uint32_t ua = (uint32_t)(A.sidx * R + s), ub = (uint32_t)(B.sidx * R + s);
                     const bool va = s < R && ua < A.sh.cnt;
@@ -683,30 +691,49 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
             const uint32_t fullA = full_bars + (uint32_t)(slotA * 8), fullB = full_bars + (uint32_t)(slotB * 8);
             BMGD_PSTAMP(1);
             bounded_mbar_wait(empty_bars + (uint32_t)(slotA * 8), parA, aborted, P);
-            __syncwarp();
+            aborted = __any_sync(0xFFFFFFFFu, aborted);
+            if (aborted) break;  // the launch has been given up: no further copies are issued
             uint32_t sent = 0;
 #pragma unroll
             for (int kk = 0; kk < kMaxBatchesPerProducer; ++kk) {
                 const int bb = b0 + kk * NPW;
-                if (bb < nbatch) sent += copy_batch(baseA, fullA, 32 * bb, rowsA[kk]);
+                if (!NULLSTEP && bb < nbatch) sent += copy_batch(baseA, fullA, 32 * bb, rowsA[kk]);
             }
             BMGD_PSTAMP(3);
             finish_stage(fullA, sent);  // a producer without a batch in this stage still counts on its barrier
+            issued_mask |= 1u << slotA;
+            issued_par = (issued_par & ~(1u << slotA)) | ((parA ^ 1u) << slotA);
             BMGD_PSTAMP(4);
             if (two) {
                 bounded_mbar_wait(empty_bars + (uint32_t)(slotB * 8), parB, aborted, P);
-                __syncwarp();
+                aborted = __any_sync(0xFFFFFFFFu, aborted);
+                if (aborted) break;
                 sent = 0;
 #pragma unroll
                 for (int kk = 0; kk < kMaxBatchesPerProducer; ++kk) {
                     const int bb = b0 + kk * NPW;
-                    if (bb < nbatch) sent += copy_batch(baseB, fullB, 32 * bb, rowsB[kk]);
+                    if (!NULLSTEP && bb < nbatch) sent += copy_batch(baseB, fullB, 32 * bb, rowsB[kk]);
                 }
                 finish_stage(fullB, sent);
+                issued_mask |= 1u << slotB;
+                issued_par = (issued_par & ~(1u << slotB)) | ((parB ^ 1u) << slotB);
                 BMGD_PSTAMP(6);
             }
         }
         cp_async_wait_all();
+        // No CTA may exit while bulk copies into its shared memory are in flight.  After a normal run the consumers
+        // have waited for every stage; after a launch that was given up they have not, so every producer warp waits
+        // here, for a bounded time, until the last phase it sent copies into has completed on each ring slot (a phase
+        // completes once all producers have arrived and all bytes have landed; if a producer gave up before arriving,
+        // the time limit ends the wait, long after the copies themselves have landed).
+        {
+            const unsigned long long t0 = global_ns();
+            for (int s = 0; s < D; ++s) {
+                if (!((issued_mask >> s) & 1u)) continue;
+                while (!mbar_try_wait(full_bars + (uint32_t)(s * 8), (issued_par >> s) & 1u))
+                    if (global_ns() - t0 > kDrainNs) break;
+            }
+        }
     } else {
         // ================================================================ consumer warps
         const int grp = lane / LPR, sub = lane % LPR;
@@ -769,7 +796,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                         __syncwarp();
                         const unsigned char* rowp = smem + plan.ring_off + cs_slot * stage_bytes + lane_off;
                         const unsigned char* yp = smem + plan.ring_off + cs_slot * stage_bytes + y_off;
-                        int nsub = min(sp_left, RB);
+                        int nsub = NULLSTEP ? 0 : min(sp_left, RB);
                         sp_left -= nsub;
                         if constexpr (NV * (int)sizeof(T) <= 32) {  // narrow rows: four independent rows in flight per group
                             for (; nsub >= 4; nsub -= 4, rowp += 4 * subpass_bytes, yp += 4 * y_step) {
@@ -974,7 +1001,9 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                         }
                     }
                     BMGD_STAMP(9);
+                    if (aborted) *cta_abort = 1;  // a thread of this CTA has given up a wait: after the barrier all consumers know
                     consumer_sync(nthreads);
+                    const int stop = *cta_abort;
                     {
                         const T* gf = gfin + sub * VEC;
 #pragma unroll
@@ -990,6 +1019,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                     }
                     BMGD_STAMP(7);
                     ++step_count;
+                    if (stop) goto consumers_done;  // the same decision in every consumer thread; theta is not written back
                 }
             }
 
@@ -1005,6 +1035,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                 }
             }
         }
+    consumers_done:;
     }
     if (S > 1) {  // no CTA leaves while a peer's packets for it may still be on their way
         __syncwarp();

@@ -253,6 +253,84 @@ def test_a_wait_that_runs_out_is_reported_and_the_handle_stays_usable():
     assert rel_l2(theta[0], want) <= 1e-4
 
 
+@pytest.mark.parametrize("shape", [
+    dict(cluster_size=4, ctas_per_chain=4),    # packets inside one cluster
+    dict(cluster_size=2, ctas_per_chain=8),    # packets between clusters too
+])  # (a lone CTA waits only on the ring's mbarriers, whose try_wait suspends in hardware and rarely fails twice)
+def test_a_step_kernel_wait_that_runs_out_ends_the_launch_and_the_handle_stays_usable(shape):
+    """The step kernel's own waits with a budget of a nanosecond: the first wait that does not succeed at its first
+    look gives up, every CTA leaves its loops (no copy left in flight, theta not written back), the next
+    synchronising call reports BMGD_ERR_TIMEOUT once, and the same handle, given a sane budget, computes correctly.
+    A wait that gives up is not a fault: nothing traps, hangs or touches memory out of bounds."""
+    from paper_2312_08728_b200.binding import Bmgd, BmgdError, ERR_TIMEOUT, FLAG_NO_SLOTS
+    w = SMALL.scaled(T=40)  # 480 steps: were the launch to run on after giving up, it would still end, only later
+    bufs = buffers_of(w)
+    X, y = [t.cuda() for t in bufs[0]]
+    with Bmgd(w.N, w.p, w.K, loss=w.loss, dtype=w.dtype, flags=FLAG_NO_SLOTS, timeout_ms=1e-6, **shape) as h:
+        start = np.full((1, w.p), 0.25, dtype=np.float32)
+        h.set_theta(start)
+        h.run_rounds_resident(X, y, w.T, w.n, w.lr, 5)
+        with pytest.raises(BmgdError) as e:
+            h.sync()
+        assert e.value.status == ERR_TIMEOUT
+        h.sync()  # reported once, then cleared
+        assert np.array_equal(h.get_theta(), start)  # the abandoned launch did not write theta back
+        h.set_timeout(0.0)  # back to the default budget
+        h.set_theta(np.zeros((1, w.p), dtype=np.float32))
+        h.run_rounds_resident(X, y, 2, w.n, w.lr, inputs.buffer_seed(w.seed, 0, 0, w.K))
+        theta = h.get_theta()
+    want = oracle_job(w.scaled(K=1, N=w.N0, T=2), bufs[:1])[0]
+    assert rel_l2(theta[0], want) <= 1e-4
+
+
+@pytest.mark.parametrize("opt", [None, "adam"])
+@pytest.mark.parametrize("shape", [dict(cluster_size=1), dict(cluster_size=4)])
+def test_more_chains_than_resident_teams(shape, opt):
+    """Rc = 200 chains on at most 148 SMs: teams take chain after chain inside one launch, the producer warps run
+    on across chain boundaries, theta and the update rule's state are reloaded per chain.  Every chain against
+    the oracle."""
+    import oracle
+    w = Workload("many-chains", LOSS_LINEAR, DTYPE_F32, N=6_000, p=24, K=1, n=500, T=2, lr=0.1, epochs=1, Rc=200,
+                 rho=0.5, seed=77)
+    bufs = buffers_of(w)
+    o = None if opt is None else dict(kind=oracle.OPT_ADAM, a=0.9, b=0.999, eps=1e-8)
+    if o:
+        w = w.scaled(lr=0.01)
+    theta, stats = gpu_job(w, bufs, mode="resident", opt=o, **shape)
+    assert stats["chains_in_flight"] < w.Rc, stats  # some team really worked on more than one chain
+    want = oracle_job(w, bufs, opt=o)
+    for c in range(w.Rc):
+        assert rel_l2(theta[c], want[c]) <= 1e-4, (c, stats)
+    assert np.unique(theta[:, 0]).size == w.Rc
+
+
+def test_null_rounds_probe_changes_nothing():
+    """The latency probe runs the step kernel's waits, exchanges and updates without rows: theta, the update
+    rule's state and the step counters stay as they are, and the handle then computes as if it had not run."""
+    from paper_2312_08728_b200.binding import Bmgd, FLAG_NO_SLOTS, FLAG_TIMING
+    import oracle
+    w = SMALL
+    bufs = buffers_of(w)
+    X, y = [t.cuda() for t in bufs[0]]
+    for shape in (dict(), dict(cluster_size=2, ctas_per_chain=8)):
+        with Bmgd(w.N, w.p, w.K, loss=w.loss, dtype=w.dtype, flags=FLAG_NO_SLOTS | FLAG_TIMING, **shape) as h:
+            h.set_optimizer(oracle.OPT_NESTEROV, 0.9)
+            h.run_rounds_resident(X, y, 1, w.n, w.lr, 3)
+            before, s0 = h.get_theta(), h.get_stats()
+            h.debug_null_rounds(X.shape[0], 5, w.n)
+            after, s1 = h.get_theta(), h.get_stats()
+            assert np.array_equal(before, after)
+            assert s1["launches"] == s0["launches"] + 1 and s1["steps"] == s0["steps"]
+            assert s1["kernel_ms"] > s0["kernel_ms"]
+            h.run_rounds_resident(X, y, 1, w.n, w.lr, 4)
+            got = h.get_theta()
+        with Bmgd(w.N, w.p, w.K, loss=w.loss, dtype=w.dtype, flags=FLAG_NO_SLOTS, **shape) as h:
+            h.set_optimizer(oracle.OPT_NESTEROV, 0.9)
+            h.run_rounds_resident(X, y, 1, w.n, w.lr, 3)
+            h.run_rounds_resident(X, y, 1, w.n, w.lr, 4)
+            assert np.array_equal(h.get_theta(), got)
+
+
 def test_algorithm_1_with_a_fresh_partition_of_the_sample_every_pass():
     """All of Algorithm 1: every pass re-partitions the sample into K buffers (host gather into pinned staging
     buffers, two in flight), every round re-partitions the buffer, theta is carried throughout."""
