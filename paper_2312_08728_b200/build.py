@@ -9,6 +9,7 @@ import subprocess
 _PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libbmgd.so")
+TRACE_LIB_PATH = os.path.join(_PKG, "libbmgd_trace.so")  # the same sources with -DBMGD_TRACE (phase clock stamps)
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -25,10 +26,10 @@ def _deps():
     return _sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(root, "include", "*.h"))
 
 
-def is_stale() -> bool:
-    if not os.path.exists(LIB_PATH):
+def is_stale(path: str = LIB_PATH) -> bool:
+    if not os.path.exists(path):
         return True
-    t = os.path.getmtime(LIB_PATH)
+    t = os.path.getmtime(path)
     return any(os.path.getmtime(f) > t for f in _deps())
 
 
@@ -39,19 +40,25 @@ def find_nvcc():
     return None
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Build libbmgd.so next to this file if it is missing or older than its sources."""
-    if not force and not is_stale():
-        return LIB_PATH
+def build(force: bool = False, verbose: bool = False, trace: bool = False) -> str:
+    """Build libbmgd.so next to this file if it is missing or older than its sources.
+
+    trace=True builds libbmgd_trace.so instead: the same sources compiled with -DBMGD_TRACE, in which thread 0 of
+    every CTA stamps the clock at the phase boundaries of its first steps (read by paper_2312_08728_b200.trace)."""
+    out = TRACE_LIB_PATH if trace else LIB_PATH
+    if not force and not is_stale(out):
+        return out
     nvcc = find_nvcc()
     if nvcc is None:
         raise RuntimeError("nvcc not found: cannot build the BMGD CUDA library")
-    tmp = LIB_PATH + f".{os.getpid()}.tmp"
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + _sources() + ["-lcudart"]
+    tmp = out + f".{os.getpid()}.tmp"
+    cmd = ([nvcc] + NVCC_FLAGS + (["-DBMGD_TRACE"] if trace else []) + (["-Xptxas", "-v"] if verbose else [])
+           + ["-o", tmp] + _sources() + ["-lcudart"])
     subprocess.check_call(cmd, cwd=CSRC)
-    os.replace(tmp, LIB_PATH)
-    return LIB_PATH
+    os.replace(tmp, out)
+    return out
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose=True))
+    import sys
+    print(build(force=True, verbose="-v" in sys.argv, trace="--trace" in sys.argv))

@@ -263,10 +263,12 @@ const GlmVariant* pick_variant(int dtype, int loss, int p, bool aligned16, int l
     return nullptr;
 }
 
-// How often a waiting thread looks at the clock and the abort flag.  A budget below a microsecond cannot be measured
-// by counting polls: then every failed poll looks, so that any wait that does not succeed at once gives up.
+// How often a waiting thread looks at the clock and the abort flag.  A budget below a microsecond cannot be measured:
+// it counts as no budget at all, and every failed poll looks, so that a wait that does not succeed at its first look
+// gives up.
 void set_poll_cadence(GlmParams* P) {
     const bool tiny = P->timeout_ns < 1000ull;
+    if (tiny) P->timeout_ns = 0;
     P->poll_mask = tiny ? 0u : 0x3FFu;
     P->mbar_mask = tiny ? 0u : 0x3Fu;
 }
@@ -1111,17 +1113,19 @@ const char* bmgd_strerror(int status) {
 int bmgd_last_cuda_error(const bmgd_t* h) { return h ? h->last_cuda : 0; }
 
 #ifdef BMGD_TRACE
-// Debug build only: copy out the clock stamps CTA 0 took at the phase boundaries of its first steps.
-int bmgd_debug_trace(long long* out_host, int count) {
-    if (!out_host || count <= 0 || count > bmgdk::kTraceSteps * bmgdk::kTracePhases) return BMGD_ERR_ARG;
-    cudaError_t e = cudaMemcpyFromSymbol(out_host, bmgdk::g_trace, sizeof(long long) * (size_t)count);
+// Debug build only: copy out the clock stamps [block][step][phase] that thread 0 of every CTA took at the phase
+// boundaries of its first steps (which = 0), or those of every CTA's first producer warp (which = 1).
+int bmgd_debug_trace(int which, long long* out_host, int count) {
+    const int total = bmgdk::kTraceBlocks * bmgdk::kTraceSteps * bmgdk::kTracePhases;
+    if (!out_host || count <= 0 || count > total || which < 0 || which > 1) return BMGD_ERR_ARG;
+    cudaError_t e = which == 0 ? cudaMemcpyFromSymbol(out_host, bmgdk::g_trace, sizeof(long long) * (size_t)count)
+                               : cudaMemcpyFromSymbol(out_host, bmgdk::g_ptrace, sizeof(long long) * (size_t)count);
     return e == cudaSuccess ? BMGD_OK : BMGD_ERR_CUDA;
 }
-// The same for the stamps of the first producer warp (indexed by the pair of ring stages it works on).
-int bmgd_debug_producer_trace(long long* out_host, int count) {
-    if (!out_host || count <= 0 || count > bmgdk::kTraceSteps * bmgdk::kTracePhases) return BMGD_ERR_ARG;
-    cudaError_t e = cudaMemcpyFromSymbol(out_host, bmgdk::g_ptrace, sizeof(long long) * (size_t)count);
-    return e == cudaSuccess ? BMGD_OK : BMGD_ERR_CUDA;
+int bmgd_debug_trace_dims(int* blocks, int* steps, int* phases) {
+    if (!blocks || !steps || !phases) return BMGD_ERR_ARG;
+    *blocks = bmgdk::kTraceBlocks; *steps = bmgdk::kTraceSteps; *phases = bmgdk::kTracePhases;
+    return BMGD_OK;
 }
 #endif
 

@@ -248,7 +248,8 @@ __host__ __device__ inline GlmSmemPlan glm_smem_plan(int warps, int gpw, bool pr
     s.stage_bytes = gathered ? s.stage_y_off + (R * elem_bytes + 127) / 128 * 128 : s.stage_y_off;
     s.ring_off = 1024;  // the stages' mbarriers sit in front of the ring
     s.ring_bytes = depth * s.stage_bytes;
-    s.gpart_rows = prereduce ? warps : warps * gpw;
+    // rounded up to a multiple of eight: the rows beyond the real ones stay zero, so the column sums need no guards
+    s.gpart_rows = ((prereduce ? warps : warps * gpw) + 7) & ~7;
     s.gpart_off = s.ring_off + s.ring_bytes;
     s.gfin_off = s.gpart_off + s.gpart_rows * pcap * elem_bytes;
     s.cpk_off = s.gfin_off + pcap * elem_bytes;
@@ -259,23 +260,23 @@ __host__ __device__ inline GlmSmemPlan glm_smem_plan(int warps, int gpw, bool pr
 }
 
 #ifdef BMGD_TRACE
-// Debug build only: clock stamps of one CTA at the phase boundaries of its first steps.
-#ifndef BMGD_TRACE_BLOCK
-#define BMGD_TRACE_BLOCK 0
-#endif
-constexpr int kTraceSteps = 64, kTracePhases = 16;
-__device__ long long g_trace[kTraceSteps * kTracePhases];
-#define BMGD_STAMP(ph)                                                                              \
-    do {                                                                                            \
-        if (blockIdx.x == BMGD_TRACE_BLOCK && threadIdx.x == 0 && step_count < (uint32_t)kTraceSteps) \
-            g_trace[step_count * kTracePhases + (ph)] = clock64();                                  \
+// Debug build only (build.py, trace=True): clock stamps of thread 0 of every CTA at the phase boundaries of its first
+// steps, and of the first producer warp per pair of ring stages.  Phase 15 of a step holds the global timer (ns) at the
+// step's start, for comparing CTAs; all other stamps are the SM's cycle counter.
+constexpr int kTraceBlocks = 64, kTraceSteps = 48, kTracePhases = 16;
+__device__ long long g_trace[kTraceBlocks * kTraceSteps * kTracePhases];
+__device__ long long g_ptrace[kTraceBlocks * kTraceSteps * kTracePhases];
+#define BMGD_STAMP(ph)                                                                                        \
+    do {                                                                                                      \
+        if (threadIdx.x == 0 && blockIdx.x < (unsigned)kTraceBlocks && step_count < (uint32_t)kTraceSteps) {    \
+            g_trace[((int)blockIdx.x * kTraceSteps + (int)step_count) * kTracePhases + (ph)] = clock64();     \
+            if ((ph) == 0) g_trace[((int)blockIdx.x * kTraceSteps + (int)step_count) * kTracePhases + 15] = (long long)global_ns(); \
+        }                                                                                                     \
     } while (0)
-// the same for the first producer warp, indexed by the pair of stages it works on
-__device__ long long g_ptrace[kTraceSteps * kTracePhases];
-#define BMGD_PSTAMP(ph)                                                                                  \
-    do {                                                                                                 \
-        if (blockIdx.x == BMGD_TRACE_BLOCK && pw == 0 && lane == 0 && (it >> 1) < (uint32_t)kTraceSteps)  \
-            g_ptrace[(it >> 1) * kTracePhases + (ph)] = clock64();                                       \
+#define BMGD_PSTAMP(ph)                                                                                       \
+    do {                                                                                                      \
+        if (pw == 0 && lane == 0 && blockIdx.x < (unsigned)kTraceBlocks && (it >> 1) < (uint32_t)kTraceSteps)   \
+            g_ptrace[((int)blockIdx.x * kTraceSteps + (int)(it >> 1)) * kTracePhases + (ph)] = clock64();     \
     } while (0)
 #else
 #define BMGD_STAMP(ph) do { } while (0)
@@ -345,7 +346,7 @@ __device__ __forceinline__ void perm_index2(uint32_t& x0, const RoundKeys& k0, u
 __device__ __forceinline__ void wait_slow_path(unsigned long long& t0, bool& aborted, const GlmParams& P) {
     const unsigned long long now = global_ns();
     if (t0 == 0) t0 = now;
-    if (now - t0 > P.timeout_ns || ((volatile int*)P.status)[1] != 0) {
+    if (now - t0 >= P.timeout_ns || ((volatile int*)P.status)[1] != 0) {
         atomicCAS(P.status, 0, kStatusTimeout);
         atomicExch(P.status + 1, 1);
         aborted = true;
@@ -368,20 +369,19 @@ __device__ __forceinline__ T gather_packets(int count, uint32_t tag, bool& abort
         unsigned long long t0 = 0;
         uint32_t spins = 0;
         while (!aborted) {
+            // no guards on the loads (a guarded load waits for the one before it): a packet index past the last one
+            // re-reads the last packet, whose tag has to match anyway
 #pragma unroll
             for (int k = 0; k < CH; ++k) {
-                if (k0 + k < count) {
+                const int kk = min(k0 + k, count - 1);
 #pragma unroll
-                    for (int w = 0; w < NW; ++w) v[k][w] = load(k0 + k, w);
-                }
+                for (int w = 0; w < NW; ++w) v[k][w] = load(kk, w);
             }
             bool ok = true;
 #pragma unroll
             for (int k = 0; k < CH; ++k) {
-                if (k0 + k < count) {
 #pragma unroll
-                    for (int w = 0; w < NW; ++w) ok &= ((uint32_t)(v[k][w] >> 32) == tag);
-                }
+                for (int w = 0; w < NW; ++w) ok &= ((uint32_t)(v[k][w] >> 32) == tag);
             }
             if (ok) break;
             if ((++spins & P.poll_mask) == 0u) wait_slow_path(t0, aborted, P);
@@ -389,26 +389,26 @@ __device__ __forceinline__ T gather_packets(int count, uint32_t tag, bool& abort
         if (!aborted) {
 #pragma unroll
             for (int k = 0; k < CH; ++k) {
-                if (k0 + k < count) {
-                    uint32_t w32[NW];
+                uint32_t w32[NW];
 #pragma unroll
-                    for (int w = 0; w < NW; ++w) w32[w] = (uint32_t)v[k][w];
-                    s += Words<T>::make(w32);
-                }
+                for (int w = 0; w < NW; ++w) w32[w] = (uint32_t)v[k][w];
+                const T val = Words<T>::make(w32);
+                s += (k0 + k < count) ? val : T(0);
             }
         }
     }
     return s;
 }
 
-// Sum `rows` values spaced `stride` elements apart, eight loads in flight at a time, fixed order.
+// Sum `rows` (a multiple of eight) values spaced `stride` elements apart, fixed order.  The loads carry no guards, so
+// that all eight of a sweep are in flight together (a guarded load waits for the one before it).
 template <typename T>
 __device__ __forceinline__ T strided_sum(const T* col, int rows, int stride) {
     T s0 = T(0), s1 = T(0);
     for (int r0 = 0; r0 < rows; r0 += 8) {
         T v[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = (r0 + j < rows) ? col[(r0 + j) * stride] : T(0);
+        for (int j = 0; j < 8; ++j) v[j] = col[(r0 + j) * stride];
         s0 += (v[0] + v[1]) + (v[2] + v[3]);
         s1 += (v[4] + v[5]) + (v[6] + v[7]);
     }
@@ -456,6 +456,61 @@ __device__ __forceinline__ void row_step(const unsigned char* rowp, const unsign
     for (int i = 0; i < NV; ++i) gacc[i] = fma(res, x[i], gacc[i]);
 }
 
+// NR rows of one group at once (rows `row_stride` bytes apart, their y values `y_stride` apart): all loads first, then
+// the NR dot products side by side, so that the latencies of the rows overlap by construction.  The gradient takes the
+// rows in ascending order, exactly as NR calls of row_step would.
+template <typename T, int VEC, int LPR, int KCH, bool LOGISTIC, int NR>
+__device__ __forceinline__ void rows_step(const unsigned char* rowp, int row_stride, const unsigned char* yp, int y_stride,
+                                          const T (&th)[KCH * VEC], T (&gacc)[KCH * VEC]) {
+    constexpr int NV = KCH * VEC;
+    constexpr int CB = VEC * (int)sizeof(T);
+    T x[NR][NV], yv[NR], dot[NR];
+#pragma unroll
+    for (int r = 0; r < NR; ++r) {
+#pragma unroll
+        for (int k = 0; k < KCH; ++k) {
+            const unsigned char* src = rowp + r * row_stride + k * LPR * CB;
+            if constexpr (CB == 16 && sizeof(T) == 4) {
+                const float4 v = *reinterpret_cast<const float4*>(src);
+                x[r][k * VEC + 0] = v.x; x[r][k * VEC + 1] = v.y; x[r][k * VEC + 2] = v.z; x[r][k * VEC + 3] = v.w;
+            } else if constexpr (CB == 16) {
+                const double2 d = *reinterpret_cast<const double2*>(src);
+                x[r][k * VEC + 0] = d.x; x[r][k * VEC + 1] = d.y;
+            } else {
+                x[r][k] = *reinterpret_cast<const T*>(src);
+            }
+        }
+        yv[r] = *reinterpret_cast<const T*>(yp + r * y_stride);
+    }
+#pragma unroll
+    for (int r = 0; r < NR; ++r) {
+        T part[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) part[e] = T(0);
+#pragma unroll
+        for (int k = 0; k < KCH; ++k)
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) part[e] = fma(x[r][k * VEC + e], th[k * VEC + e], part[e]);
+        dot[r] = part[0];
+#pragma unroll
+        for (int e = 1; e < VEC; ++e) dot[r] += part[e];
+    }
+#pragma unroll
+    for (int off = LPR / 2; off > 0; off >>= 1)
+#pragma unroll
+        for (int r = 0; r < NR; ++r) dot[r] += __shfl_xor_sync(0xFFFFFFFFu, dot[r], off);
+    T res[NR];
+#pragma unroll
+    for (int r = 0; r < NR; ++r) {
+        if constexpr (LOGISTIC) res[r] = sigmoid_of(dot[r]) - yv[r];
+        else res[r] = dot[r] - yv[r];
+    }
+#pragma unroll
+    for (int i = 0; i < NV; ++i)
+#pragma unroll
+        for (int r = 0; r < NR; ++r) gacc[i] = fma(res[r], x[r][i], gacc[i]);
+}
+
 // Waits for a phase of an mbarrier in this CTA's shared memory with the kernel's bounded-wait protocol.
 __device__ __forceinline__ void bounded_mbar_wait(uint32_t bar, uint32_t parity, bool& aborted, const GlmParams& P) {
     unsigned long long t0 = 0;
@@ -493,6 +548,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
     constexpr bool G4 = glm_gathered(CB, PCAP);  // rows arrive four at a time through the tensor map `xmap` of X
     constexpr int YOFF = PCAP * (int)sizeof(T);  // other layouts: y sits behind the predictors of its row
     constexpr uint32_t kNoRow = 0xFFFFFFFFu;
+    constexpr int kClusterChunk = (sizeof(T) == 4 && MAXT <= kGlmSmallCta) ? 8 : 4;  // packets of the cluster's CTAs read per sweep of a poll
 
     extern __shared__ __align__(1024) unsigned char smem[];  // gathers want 128-byte aligned destinations
 
@@ -748,9 +804,21 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
         const int y_step = G4 ? spp * (int)sizeof(T) : subpass_bytes;
         const uint32_t warp_first = (uint32_t)(warp * GPW);  // first row slot of this warp in sub-pass 0
         const int slice = (p + S - 1) / S;  // predictors owned by one CTA of a cluster in the sliced exchange
+        // Pushing one predictor's sum to all S peers is a run of S dependent remote stores in one thread.  Where the
+        // consumer threads outnumber the predictors, xg_n threads share the pushes of a predictor: thread (xf, xg) sends
+        // predictor xf to peers xg, xg + xg_n, ...  (each of them sums the CTA's partial rows for xf itself).
+        int fw_log2 = 5;  // predictors rounded up to a power of two of at least a warp
+        while ((1 << fw_log2) < p) ++fw_log2;
+        // threads that share a predictor's pushes: a power of two, at most S (cluster sizes are powers of two)
+        const int xg_n = (FPT == 1 && cpc == 1 && S > 1) ? max(1, min(S, nthreads >> fw_log2)) : 1;
+        const int xf = (xg_n > 1) ? (tid & ((1 << fw_log2) - 1)) : tid, xg = (xg_n > 1) ? (tid >> fw_log2) : 0;
         const T scale_full = (T)P.scale_full, scale_last = (T)P.scale_last;
         const T inv_full = (T)P.inv_full, inv_last = (T)P.inv_last, lr_const = (T)P.lr;
 
+        // A full mini-batch is dealt to the CTAs the same way in every step: its share, and the sub-passes in which this
+        // warp has rows, are worked out once (the divisions would otherwise sit at the head of every step).
+        const RowShare share_full = row_share(0u, n, n, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full);
+        const int sp_full = (share_full.cnt > warp_first) ? (int)((share_full.cnt - warp_first - 1u) / (uint32_t)spp) + 1 : 0;
         int cs_slot = 0;         // ring slot the compute cursor reads next
         uint32_t cs_phase = 0;   // parity of that slot's "full" phase
         uint32_t step_count = 0; // steps this team has finished in this launch
@@ -782,7 +850,10 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
 
             for (int t = 0; t < T_rounds; ++t) {
                 for (uint32_t m = 0; m < M; ++m) {
-                    const RowShare sh = row_share(m, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full);
+                    const bool full_batch = m * n + n <= N0;
+                    RowShare sh = share_full;
+                    sh.lo = m * n;
+                    if (!full_batch) sh = row_share(m, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full);
                     BMGD_STAMP(0);
 
                     T gacc[NV];
@@ -790,25 +861,27 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                     for (int i = 0; i < NV; ++i) gacc[i] = T(0);
 
                     // sub-passes of this step in which the warp has at least one row
-                    int sp_left = (sh.cnt > warp_first) ? (int)((sh.cnt - warp_first - 1u) / (uint32_t)spp) + 1 : 0;
+                    int sp_left = sp_full;
+                    if (!full_batch) sp_left = (sh.cnt > warp_first) ? (int)((sh.cnt - warp_first - 1u) / (uint32_t)spp) + 1 : 0;
                     for (int sidx = 0; sidx < passes; ++sidx) {
                         bounded_mbar_wait(full_bars + (uint32_t)(cs_slot * 8), cs_phase, aborted, P);
                         __syncwarp();
+                        if (sidx == 0) BMGD_STAMP(10);
                         const unsigned char* rowp = smem + plan.ring_off + cs_slot * stage_bytes + lane_off;
                         const unsigned char* yp = smem + plan.ring_off + cs_slot * stage_bytes + y_off;
                         int nsub = NULLSTEP ? 0 : min(sp_left, RB);
                         sp_left -= nsub;
                         if constexpr (NV * (int)sizeof(T) <= 32) {  // narrow rows: four independent rows in flight per group
-                            for (; nsub >= 4; nsub -= 4, rowp += 4 * subpass_bytes, yp += 4 * y_step) {
-                                row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, yp, th, gacc);
-                                row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + subpass_bytes, yp + y_step, th, gacc);
-                                row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + 2 * subpass_bytes, yp + 2 * y_step, th, gacc);
-                                row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + 3 * subpass_bytes, yp + 3 * y_step, th, gacc);
-                            }
+                            for (; nsub >= 4; nsub -= 4, rowp += 4 * subpass_bytes, yp += 4 * y_step)
+                                rows_step<T, VEC, LPR, KCH, LOGISTIC, 4>(rowp, subpass_bytes, yp, y_step, th, gacc);
                         }
                         for (; nsub >= 2; nsub -= 2, rowp += 2 * subpass_bytes, yp += 2 * y_step) {  // two independent rows in flight per group
-                            row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, yp, th, gacc);
-                            row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + subpass_bytes, yp + y_step, th, gacc);
+                            if constexpr (NV <= 16) {
+                                rows_step<T, VEC, LPR, KCH, LOGISTIC, 2>(rowp, subpass_bytes, yp, y_step, th, gacc);
+                            } else {  // wide per-lane state: two rows' values at once would not fit the registers
+                                row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, yp, th, gacc);
+                                row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp + subpass_bytes, yp + y_step, th, gacc);
+                            }
                         }
                         if (nsub) row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, yp, th, gacc);
                         __syncwarp();  // every lane has its values in registers: the slot may be refilled
@@ -842,8 +915,8 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                     T tot[FPT];
 #pragma unroll
                     for (int i = 0; i < FPT; ++i) {
-                        const int f = tid + i * nthreads;
-                        tot[i] = (f < p) ? strided_sum(gpart + f, plan.gpart_rows, PCAP) : T(0);
+                        const int f = xf + i * nthreads;  // xf == tid unless this thread helps with another thread's pushes
+                        tot[i] = (f < p && xg < xg_n) ? strided_sum(gpart + f, plan.gpart_rows, PCAP) : T(0);
                     }
                     BMGD_STAMP(3);
 
@@ -860,13 +933,13 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                         if (S > 1) {
     #pragma unroll
                             for (int i = 0; i < FPT; ++i) {
-                                const int f = tid + i * nthreads;
-                                if (f < p) {
+                                const int f = xf + i * nthreads;
+                                if (f < p && xg < xg_n) {
     #pragma unroll
                                     for (int w = 0; w < NW; ++w) {
                                         const unsigned long long pk = ((unsigned long long)tag << 32) | Words<T>::get(tot[i], w);
                                         const uint32_t mine = cpk + (uint32_t)((rank * plan.cpk_stride + f * NW + w) * 8);
-                                        for (int peer = 0; peer < S; ++peer) st_cluster_u64(map_to_cta(mine, (uint32_t)peer), pk);
+                                        for (int peer = xg; peer < S; peer += xg_n) st_cluster_u64(map_to_cta(mine, (uint32_t)peer), pk);
                                     }
                                 }
                             }
@@ -875,7 +948,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                             for (int i = 0; i < FPT; ++i) {
                                 const int f = tid + i * nthreads;
                                 if (f < p)
-                                    tot[i] = gather_packets<T, kMaxClusterSize, 4>(
+                                    tot[i] = gather_packets<T, kMaxClusterSize, kClusterChunk>(
                                         S, tag, aborted, P,
                                         [&](int k, int w) { return ld_shared_volatile_u64(cpk + (uint32_t)((k * plan.cpk_stride + f * NW + w) * 8)); });
                             }
@@ -910,7 +983,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                             const int f = rank * slice + j;
                             if (j < slice && f < p) {
                                 const T mine_sum = (S > 1)
-                                    ? gather_packets<T, kMaxClusterSize, 4>(
+                                    ? gather_packets<T, kMaxClusterSize, kClusterChunk>(
                                           S, tag, aborted, P,
                                           [&](int k, int w) { return ld_shared_volatile_u64(cpk + (uint32_t)((k * plan.cpk_stride + j * NW + w) * 8)); })
                                     : tot[i];
@@ -928,7 +1001,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                             if (j >= slice || f >= p) continue;
                             const unsigned long long* src = slot + f * NW;
                             const int stride = P.ll_stride;
-                            const T s = gather_packets<T, kMaxCpc, kMaxCpc>(
+                            const T s = gather_packets<T, kMaxCpc, 4>(
                                 cpc, tag, aborted, P, [&](int k, int w) { return ld_packet(src + (size_t)k * stride + w); });
                             if (S > 1) {
     #pragma unroll
@@ -958,7 +1031,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                     // ---- the thread that holds predictor f's gradient sum applies the update rule to its master copy of
                     //      theta_f (the same arithmetic in every CTA, so all copies stay bit-identical) and publishes it;
                     //      then every lane refreshes the coefficients it multiplies rows with
-                    const bool full = min(n, N0 - sh.lo) == n;
+                    const bool full = full_batch;
                     T lr = lr_const;
                     if (P.sched == kLrCosine) {  // Section 4.4: rate of the j-th update of a pass of J updates
                         const long long j = sched_pos + 1;
