@@ -45,6 +45,8 @@ def lib() -> ctypes.CDLL:
         L.orc_round_keys.restype = None
         L.orc_perm_index.argtypes = [ctypes.c_uint32, ctypes.c_uint32, u32p]
         L.orc_perm_index.restype = ctypes.c_uint32
+        L.orc_domain.argtypes = [ctypes.c_uint32, u32p, u32p]
+        L.orc_domain.restype = None
         L.orc_perm.argtypes = [ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_void_p]
         L.orc_perm.restype = None
         L.orc_run_rounds.argtypes = [
@@ -73,6 +75,13 @@ def round_keys(seed: int, chain: int, rnd: int):
     out = (ctypes.c_uint32 * 8)()
     lib().orc_round_keys(int(seed) & 0xFFFFFFFFFFFFFFFF, chain, rnd, out)
     return [int(v) for v in out]
+
+
+def domain(N0: int):
+    """(a, c): the sizes of the two halves of the Feistel network for a buffer of N0 rows."""
+    a, c = ctypes.c_uint32(), ctypes.c_uint32()
+    lib().orc_domain(N0, ctypes.byref(a), ctypes.byref(c))
+    return a.value, c.value
 
 
 def perm(seed: int, chain: int, rnd: int, N0: int) -> np.ndarray:

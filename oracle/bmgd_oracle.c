@@ -28,9 +28,9 @@
  *
  * The bijection: round keys come from the Philox4x32-10 counter-based generator
  * (Salmon, Moraes, Dror, Shaw, SC'11), counter = (round, chain, tag, block), key = seed;
- * the keys drive an 8-round alternating unbalanced Feistel network on
- * b = max(10, ceil(log2 N0)) bits, and values >= N0 are walked round the cycle until
- * they fall below N0.
+ * the keys drive an 8-round alternating Feistel network with modular addition on
+ * Z_a x Z_c, a = max(32, ceil(sqrt(N0))), c = max(32, ceil(N0 / a)), so that a c >= N0 is
+ * barely larger than N0; values >= N0 are walked round the cycle until they fall below N0.
  *
  * All floating point is fp64.  Stored inputs (fp64, fp32 or bf16) are widened exactly.
  * Threads (OpenMP, optional) split rows for the residuals and columns for the gradient,
@@ -90,10 +90,10 @@ void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t ou
 /* ------------------------------------------------------------------ shuffle */
 
 #define ORC_SHUFFLE_TAG 0x424D4744u /* "BMGD" */
-/* Narrow Feistel halves (3 bits and below) fail the chi-square gate on mini-batch
- * co-membership, so the network never works on fewer than 10 bits; small buffers
- * just walk the cycle longer. */
-#define ORC_MIN_BITS 10u
+/* Narrow Feistel halves fail the chi-square gate on mini-batch co-membership, so neither
+ * half of the network is ever smaller than 32 values; small buffers just walk the cycle
+ * longer. */
+#define ORC_MIN_HALF 32u
 
 /* Eight Feistel round keys for (seed, chain, round). */
 void orc_round_keys(uint64_t seed, uint32_t chain, uint32_t round, uint32_t keys[8]) {
@@ -104,34 +104,44 @@ void orc_round_keys(uint64_t seed, uint32_t chain, uint32_t round, uint32_t keys
     orc_philox4x32_10(ctr, key, keys + 4);
 }
 
-static uint32_t ceil_log2_u32(uint32_t v) {
-    uint32_t b = 0;
-    while (b < 32 && ((uint64_t)1 << b) < (uint64_t)v) ++b;
-    return b;
+/* The two halves of the network for a buffer of N0 rows: a = max(32, ceil(sqrt(N0))) values
+ * in the high half, c = max(32, ceil(N0 / a)) in the low half.  a c >= N0, and for
+ * N0 >= 1024 the excess a c - N0 is below a, i.e. a fraction of about 1/sqrt(N0). */
+void orc_domain(uint32_t N0, uint32_t *a_out, uint32_t *c_out) {
+    uint32_t a = (uint32_t)sqrt((double)N0);
+    while ((uint64_t)a * a < N0) ++a;                       /* smallest a with a^2 >= N0 */
+    while (a > 0 && (uint64_t)(a - 1) * (a - 1) >= N0) --a;
+    if (a < ORC_MIN_HALF) a = ORC_MIN_HALF;
+    uint32_t c = (uint32_t)(((uint64_t)N0 + a - 1) / a);
+    if (c < ORC_MIN_HALF) c = ORC_MIN_HALF;
+    *a_out = a;
+    *c_out = c;
 }
 
-static uint32_t feistel_f(uint32_t v, uint32_t k) {
+/* Round function: a keyed 32-bit hash of the other half, scaled into [0, m). */
+static uint32_t feistel_g(uint32_t v, uint32_t k, uint32_t m) {
     uint32_t hi, lo;
     mulhilo32(0xD2511F53u, v + k, &hi, &lo);
-    return hi ^ lo;
+    uint32_t f = hi ^ lo;
+    return (uint32_t)(((uint64_t)f * (uint64_t)m) >> 32);  /* floor(f m / 2^32) */
 }
 
-/* pi(j) for j in [0, N0). */
+/* pi(j) for j in [0, N0).  A value x of the network's domain [0, a c) is the pair
+ * (L, R) = (x div c, x mod c).  Each round adds, modulo the size of one half, a function of
+ * the other half: invertible, so the eight rounds are a bijection of [0, a c), and walking
+ * the cycle until the value is below N0 makes it a bijection of [0, N0). */
 uint32_t orc_perm_index(uint32_t j, uint32_t N0, const uint32_t keys[8]) {
-    uint32_t b = ceil_log2_u32(N0);
-    if (b < ORC_MIN_BITS) b = ORC_MIN_BITS;
-    uint32_t a = b / 2, c = b - a;
-    uint32_t maskA = (a >= 32) ? 0xFFFFFFFFu : (((uint32_t)1 << a) - 1u);
-    uint32_t maskC = (c >= 32) ? 0xFFFFFFFFu : (((uint32_t)1 << c) - 1u);
+    uint32_t a, c;
+    orc_domain(N0, &a, &c);
     uint32_t x = j;
     do {
-        uint32_t L = x >> c;
-        uint32_t R = x & maskC;
+        uint32_t L = x / c;
+        uint32_t R = x % c;
         for (int r = 0; r < 8; ++r) {
-            if ((r & 1) == 0) L ^= feistel_f(R, keys[r]) & maskA;
-            else              R ^= feistel_f(L, keys[r]) & maskC;
+            if ((r & 1) == 0) L = (L + feistel_g(R, keys[r], a)) % a;
+            else              R = (R + feistel_g(L, keys[r], c)) % c;
         }
-        x = (L << c) | R;
+        x = L * c + R;
     } while (x >= N0);
     return x;
 }

@@ -322,22 +322,21 @@ __device__ __forceinline__ RowShare row_share(uint32_t m, uint32_t n, uint32_t N
 }
 
 // Two indices through the shuffle at once, each under its own round keys: the two Feistel chains are independent,
-// so their latencies overlap.
+// so their latencies overlap.  Nearly every index leaves the network below N0 after one pass.
 __device__ __forceinline__ void perm_index2(uint32_t& x0, const RoundKeys& k0, uint32_t& x1, const RoundKeys& k1,
                                             const FeistelDomain& d) {
     bool w0 = true, w1 = true;  // still walking the cycle
     do {
-        uint32_t L0 = x0 >> d.c, R0 = x0 & d.maskC;
-        uint32_t L1 = x1 >> d.c, R1 = x1 & d.maskC;
+        uint32_t L0, R0, L1, R1;
+        feistel_split(x0, d, L0, R0);
+        feistel_split(x1, d, L1, R1);
 #pragma unroll
         for (int r = 0; r < 8; r += 2) {
-            L0 ^= feistel_f(R0, k0.k[r]) & d.maskA;
-            L1 ^= feistel_f(R1, k1.k[r]) & d.maskA;
-            R0 ^= feistel_f(L0, k0.k[r + 1]) & d.maskC;
-            R1 ^= feistel_f(L1, k1.k[r + 1]) & d.maskC;
+            feistel_round_pair(L0, R0, k0.k[r], k0.k[r + 1], d);
+            feistel_round_pair(L1, R1, k1.k[r], k1.k[r + 1], d);
         }
-        if (w0) { x0 = (L0 << d.c) | R0; w0 = x0 >= d.N0; }
-        if (w1) { x1 = (L1 << d.c) | R1; w1 = x1 >= d.N0; }
+        if (w0) { x0 = L0 * d.c + R0; w0 = x0 >= d.N0; }
+        if (w1) { x1 = L1 * d.c + R1; w1 = x1 >= d.N0; }
     } while (w0 || w1);
 }
 

@@ -6,9 +6,13 @@
 //
 //   round keys  k0..k7 = two blocks of Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11) with
 //               counter (t, c, 'BMGD', block) and key (seed_lo, seed_hi);
-//   bijection   eight rounds of an alternating unbalanced Feistel network on
-//               b = max(10, ceil(log2 N0)) bits, round function F(v, k) = hi ^ lo of
-//               0xD2511F53 * (v + k); outputs >= N0 are fed back in until one is < N0.
+//   bijection   a value x of [0, a c) is the pair (L, R) = (x div c, x mod c), with
+//               a = max(32, ceil(sqrt N0)) and c = max(32, ceil(N0 / a)): the smallest near-square
+//               grid that holds N0, so that almost every x is below N0.  Eight rounds alternate
+//               L <- (L + G(R, k, a)) mod a  and  R <- (R + G(L, k, c)) mod c, where
+//               G(v, k, m) = floor(F m / 2^32) and F = hi ^ lo of 0xD2511F53 * (v + k mod 2^32);
+//               outputs >= N0 (a fraction of about 1/sqrt(N0)) are fed back in until one is < N0.
+//               Each round is invertible, so pi is a bijection of [0, N0) for every key.
 //
 // The same bijection, over the whole sample of N rows with the chain word 0xFFFFFFFF and the pass number as
 // the round word, is the partition of the sample into buffers that Algorithm 1 draws at the top of each
@@ -25,21 +29,28 @@ struct RoundKeys {
 
 struct FeistelDomain {
     uint32_t N0;
-    uint32_t c;      // low-half width in bits
-    uint32_t maskA;  // high half
-    uint32_t maskC;  // low half
+    uint32_t a;      // values of the high half
+    uint32_t c;      // values of the low half
+    uint32_t inv_c;  // ceil(2^32 / c): turns the division by c into a multiplication
 };
 
 __host__ __device__ inline FeistelDomain make_domain(uint32_t N0) {
-    uint32_t b = 0;
-    while (b < 32 && (1ull << b) < (unsigned long long)N0) ++b;
-    if (b < 10) b = 10;
-    const uint32_t a = b >> 1, c = b - a;
+    // floor(sqrt(N0 - 1)) bit by bit; one more is the smallest a with a * a >= N0
+    const uint32_t v = N0 > 0 ? N0 - 1u : 0u;
+    uint32_t root = 0;
+    for (int bit = 15; bit >= 0; --bit) {
+        const uint32_t t = root | (1u << bit);
+        if ((unsigned long long)t * t <= (unsigned long long)v) root = t;
+    }
+    uint32_t a = root + 1u;
+    if (a < 32u) a = 32u;
+    uint32_t c = (uint32_t)(((unsigned long long)N0 + a - 1u) / a);
+    if (c < 32u) c = 32u;
     FeistelDomain d;
     d.N0 = N0;
+    d.a = a;
     d.c = c;
-    d.maskA = (1u << a) - 1u;            // a <= 16
-    d.maskC = (c >= 32) ? 0xFFFFFFFFu : ((1u << c) - 1u);
+    d.inv_c = (uint32_t)(0xFFFFFFFFull / c) + 1u;  // c >= 32, so this fits 32 bits
     return d;
 }
 
@@ -75,23 +86,40 @@ __host__ __device__ __forceinline__ RoundKeys round_keys(uint64_t seed, uint32_t
     return rk;
 }
 
-__host__ __device__ __forceinline__ uint32_t feistel_f(uint32_t v, uint32_t k) {
+// keyed 32-bit hash of one half, scaled into [0, m)
+__host__ __device__ __forceinline__ uint32_t feistel_g(uint32_t v, uint32_t k, uint32_t m) {
     // one 32 x 32 -> 64 bit multiply gives both halves
     const unsigned long long pr = (unsigned long long)0xD2511F53u * (unsigned long long)(uint32_t)(v + k);
-    return (uint32_t)(pr >> 32) ^ (uint32_t)pr;
+    return mulhi32((uint32_t)(pr >> 32) ^ (uint32_t)pr, m);
+}
+
+// x -> (x div c, x mod c) for x < a c < 2^32.  mulhi(x, ceil(2^32 / c)) is the quotient or one more (the rounding up
+// of the reciprocal adds less than one to x / c); one more shows as a remainder that wrapped round.
+__host__ __device__ __forceinline__ void feistel_split(uint32_t x, const FeistelDomain& d, uint32_t& L, uint32_t& R) {
+    uint32_t q = mulhi32(x, d.inv_c);
+    uint32_t r = x - q * d.c;
+    if (r >= d.c) { q -= 1u; r += d.c; }
+    L = q;
+    R = r;
+}
+
+// two rounds of the network: both halves are below their moduli before and after
+__host__ __device__ __forceinline__ void feistel_round_pair(uint32_t& L, uint32_t& R, uint32_t k_even, uint32_t k_odd,
+                                                            const FeistelDomain& d) {
+    L += feistel_g(R, k_even, d.a);
+    if (L >= d.a) L -= d.a;
+    R += feistel_g(L, k_odd, d.c);
+    if (R >= d.c) R -= d.c;
 }
 
 __host__ __device__ __forceinline__ uint32_t perm_index(uint32_t j, const FeistelDomain& d, const RoundKeys& rk) {
     uint32_t x = j;
     do {
-        uint32_t L = x >> d.c;
-        uint32_t R = x & d.maskC;
+        uint32_t L, R;
+        feistel_split(x, d, L, R);
 #pragma unroll
-        for (int r = 0; r < 8; r += 2) {
-            L ^= feistel_f(R, rk.k[r]) & d.maskA;
-            R ^= feistel_f(L, rk.k[r + 1]) & d.maskC;
-        }
-        x = (L << d.c) | R;
+        for (int r = 0; r < 8; r += 2) feistel_round_pair(L, R, rk.k[r], rk.k[r + 1], d);
+        x = L * d.c + R;
     } while (x >= d.N0);
     return x;
 }

@@ -100,6 +100,30 @@ def test_perm_is_a_bijection_at_workload_sizes(N0):
     assert int(seen.sum()) == N0
 
 
+def test_domain_is_the_smallest_near_square_grid_that_holds_the_buffer():
+    """a = max(32, ceil(sqrt N0)), c = max(32, ceil(N0 / a)), checked with exact integer arithmetic: the grid holds
+    every index, and (beyond the floor of 32 per half) drops fewer than a of its a c values."""
+    import math
+    sizes = list(range(1, 3000)) + [4095, 4096, 4097, 99_999, 100_000, 100_001, 1_000_000, 2_500_000,
+                                    46_340 ** 2, 46_340 ** 2 + 1, 2 ** 31 - 1]
+    for N0 in sizes:
+        a, c = oracle.domain(N0)
+        r = math.isqrt(N0 - 1) + 1 if N0 > 1 else 1      # smallest integer whose square is >= N0
+        assert a == max(32, r), N0
+        assert c == max(32, -(-N0 // a)), N0
+        assert a * c >= N0 and a * c < 2 ** 32
+        if N0 >= 1024:
+            assert a * c - N0 < a, N0
+
+
+def test_almost_no_index_walks_the_cycle_at_workload_sizes():
+    """With a c barely above N0, the share of indices whose first pass through the network lands at or above N0 is
+    about (a c - N0) / (a c): the walk that makes the bijection exact is rare, not the common case."""
+    for N0 in (100_000, 1_000_000, 2_500_000):
+        a, c = oracle.domain(N0)
+        assert (a * c - N0) / (a * c) < 2e-3
+
+
 def test_perm_index_agrees_with_whole_perm():
     N0 = 777
     ks = oracle.round_keys(9, 2, 5)
