@@ -261,8 +261,7 @@ __host__ __device__ inline GlmSmemPlan glm_smem_plan(int warps, int gpw, bool pr
 
 #ifdef BMGD_TRACE
 // Debug build only (build.py, trace=True): clock stamps of thread 0 of every CTA at the phase boundaries of its first
-// steps, and of the first producer warp per pair of ring stages.  Phase 15 of a step holds the global timer (ns) at the
-// step's start, for comparing CTAs; all other stamps are the SM's cycle counter.
+// steps, and of the first producer warp per pair of ring stages: the SM's cycle counter.
 constexpr int kTraceBlocks = 64, kTraceSteps = 48, kTracePhases = 16;
 __device__ long long g_trace[kTraceBlocks * kTraceSteps * kTracePhases];
 __device__ long long g_ptrace[kTraceBlocks * kTraceSteps * kTracePhases];
@@ -270,7 +269,6 @@ __device__ long long g_ptrace[kTraceBlocks * kTraceSteps * kTracePhases];
     do {                                                                                                      \
         if (threadIdx.x == 0 && blockIdx.x < (unsigned)kTraceBlocks && step_count < (uint32_t)kTraceSteps) {    \
             g_trace[((int)blockIdx.x * kTraceSteps + (int)step_count) * kTracePhases + (ph)] = clock64();     \
-            if ((ph) == 0) g_trace[((int)blockIdx.x * kTraceSteps + (int)step_count) * kTracePhases + 15] = (long long)global_ns(); \
         }                                                                                                     \
     } while (0)
 #define BMGD_PSTAMP(ph)                                                                                       \
@@ -811,6 +809,18 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
         // threads that share a predictor's pushes: a power of two, at most S (cluster sizes are powers of two)
         const int xg_n = (FPT == 1 && cpc == 1 && S > 1) ? max(1, min(S, nthreads >> fw_log2)) : 1;
         const int xf = (xg_n > 1) ? (tid & ((1 << fw_log2) - 1)) : tid, xg = (xg_n > 1) ? (tid >> fw_log2) : 0;
+        // Where this thread's packets go in its peers' shared memory (parity 0; the other parity lies a fixed distance
+        // behind), worked out once when a thread has at most four peers to serve: the address arithmetic and the mapping
+        // into the peer's window would otherwise be redone in every step, on the path from one theta to the next.
+        constexpr int kFastPeers = 4;
+        const int my_peers = (S + xg_n - 1 - xg) / xg_n;  // peers xg, xg + xg_n, ... below S
+        const bool fast_push = FPT == 1 && cpc == 1 && S > 1 && S / xg_n <= kFastPeers;
+        uint32_t push_addr[kFastPeers];
+#pragma unroll
+        for (int i = 0; i < kFastPeers; ++i)
+            push_addr[i] = (fast_push && i < my_peers)
+                ? map_to_cta(cpk_base + (uint32_t)((rank * plan.cpk_stride + xf * NW) * 8), (uint32_t)(xg + i * xg_n)) : 0u;
+        const uint32_t parity_bytes = (uint32_t)(S * plan.cpk_stride * 8);
         const T scale_full = (T)P.scale_full, scale_last = (T)P.scale_last;
         const T inv_full = (T)P.inv_full, inv_last = (T)P.inv_last, lr_const = (T)P.lr;
 
@@ -930,15 +940,28 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                         //      shared memory of every CTA of the cluster and then sums, in rank order, the S packets per
                         //      predictor that arrive in its own.  No cluster barrier: a packet is its own flag.
                         if (S > 1) {
-    #pragma unroll
-                            for (int i = 0; i < FPT; ++i) {
-                                const int f = xf + i * nthreads;
-                                if (f < p && xg < xg_n) {
+                            if (fast_push) {
+                                if (xf < p && xg < xg_n) {
+                                    const uint32_t poff = parity ? parity_bytes : 0u;
     #pragma unroll
                                     for (int w = 0; w < NW; ++w) {
-                                        const unsigned long long pk = ((unsigned long long)tag << 32) | Words<T>::get(tot[i], w);
-                                        const uint32_t mine = cpk + (uint32_t)((rank * plan.cpk_stride + f * NW + w) * 8);
-                                        for (int peer = xg; peer < S; peer += xg_n) st_cluster_u64(map_to_cta(mine, (uint32_t)peer), pk);
+                                        const unsigned long long pk = ((unsigned long long)tag << 32) | Words<T>::get(tot[0], w);
+    #pragma unroll
+                                        for (int i = 0; i < kFastPeers; ++i)
+                                            if (i < my_peers) st_cluster_u64(push_addr[i] + poff + (uint32_t)(w * 8), pk);
+                                    }
+                                }
+                            } else {
+    #pragma unroll
+                                for (int i = 0; i < FPT; ++i) {
+                                    const int f = xf + i * nthreads;
+                                    if (f < p && xg < xg_n) {
+    #pragma unroll
+                                        for (int w = 0; w < NW; ++w) {
+                                            const unsigned long long pk = ((unsigned long long)tag << 32) | Words<T>::get(tot[i], w);
+                                            const uint32_t mine = cpk + (uint32_t)((rank * plan.cpk_stride + f * NW + w) * 8);
+                                            for (int peer = xg; peer < S; peer += xg_n) st_cluster_u64(map_to_cta(mine, (uint32_t)peer), pk);
+                                        }
                                     }
                                 }
                             }

@@ -92,10 +92,6 @@ def trace_workload(L, spec):
     for label, a, b in (PHASES_MULTI if multi else PHASES_ONE):
         d = np.median(t[:nblk, steps, b] - t[:nblk, steps, a], axis=1)
         print(f"   {label:18s} {int(d[0]):6d}   (CTAs: min {int(d.min()):6d}  median {int(np.median(d)):6d}  max {int(d.max()):6d})")
-    # how far apart the CTAs of CTA 0's team start a step, by the global timer (ns)
-    team = min(nblk, st["ctas_per_chain"])
-    g = t[:team, steps, 15]
-    print(f"   step start, latest minus earliest CTA of the team (global timer): median {int(np.median(g.max(axis=0) - g.min(axis=0)))} ns")
     pt = read_stamps(L, 1)
     for label, a, b in PRODUCER:
         d = np.median(pt[:nblk, steps, b] - pt[:nblk, steps, a], axis=1)
