@@ -110,7 +110,6 @@ int validate(const bmgd_config* c) {
     if (c->loss == BMGD_LOSS_SOFTMAX) {
         if (c->C < 2 || c->C > 16) return c->C < 2 ? BMGD_ERR_ARG : BMGD_ERR_UNIMPLEMENTED;
         if (c->dtype != BMGD_BF16X_F32W) return BMGD_ERR_UNIMPLEMENTED;
-        if (c->Rc != 1) return BMGD_ERR_UNIMPLEMENTED;
     } else {
         if (c->C != 1) return BMGD_ERR_ARG;
         if (c->dtype == BMGD_BF16X_F32W) return BMGD_ERR_UNIMPLEMENTED;
@@ -120,7 +119,7 @@ int validate(const bmgd_config* c) {
     for (int i = 0; i < 4; ++i)
         if (c->reserved[i] != 0) return BMGD_ERR_ARG;
     if (c->first_chain < 0 || (int64_t)c->first_chain + c->Rc > 0x7FFFFFFFll) return BMGD_ERR_ARG;
-    if (c->first_chain != 0 && c->loss == BMGD_LOSS_SOFTMAX) return BMGD_ERR_UNIMPLEMENTED;
+
     if (c->lanes_per_row != 0 && c->lanes_per_row != 4 && c->lanes_per_row != 8 && c->lanes_per_row != 16 &&
         c->lanes_per_row != 32)
         return BMGD_ERR_ARG;
@@ -565,47 +564,51 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
     return BMGD_OK;
 }
 
+int run_softmax(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, int n, double lr, uint64_t seed, bool null_step) {
+    bmgdk::SoftmaxLaunchInfo info{};
+    EventPair ep{};
+    const bool timing = (h->cfg.flags & BMGD_FLAG_TIMING) != 0;
+    if (timing) {
+        int rc = take_events(h, &ep);
+        if (rc != BMGD_OK) return rc;
+        BMGD_CUDA(h, cudaEventRecord(ep.a, h->compute));
+    }
+    int rc = bmgdk::softmax_run(dx, dy, rows, h->cfg.p, h->cfg.C, h->cfg.Rc, (uint32_t)h->cfg.first_chain, h->base + h->lay.theta,
+                               reinterpret_cast<int*>(h->base + h->lay.status), rounds, n, lr, seed,
+                               (h->cfg.flags & BMGD_FLAG_FIXED_PARTITION) ? 1 : 0, h->timeout_ns, h->cfg.cluster_size,
+                               (h->cfg.flags & BMGD_FLAG_SOFTMAX_CUDA_CORES) ? 1 : 0, null_step ? 1 : 0, h->smem_optin,
+                               h->compute, &info);
+    if (rc != BMGD_OK) {
+        if (info.cuda_error) h->last_cuda = info.cuda_error;
+        if (timing) h->event_pool.push_back(ep);
+        return rc;
+    }
+    if (timing) {
+        BMGD_CUDA(h, cudaEventRecord(ep.b, h->compute));
+        h->kernel_events.push_back(ep);
+    }
+    const int64_t M = (rows + n - 1) / n;
+    h->stats.launches += info.launches;
+    if (!null_step) {
+        h->stats.steps += (int64_t)h->cfg.Rc * rounds * M;
+        h->stats.sample_grads += (int64_t)h->cfg.Rc * rounds * rows;
+    }
+    h->stats.grid_ctas = info.grid_ctas;
+    h->stats.cluster_size = info.cluster_size;
+    h->stats.ctas_per_chain = info.cluster_size;
+    h->stats.threads_per_cta = info.threads;
+    h->stats.pipeline_depth = info.depth;
+    h->stats.subpasses_per_stage = 0;
+    h->stats.smem_bytes = info.smem;
+    h->stats.chains_in_flight = info.chains_in_flight;
+    return BMGD_OK;
+}
+
 int run_any(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, int n, double lr, uint64_t seed) {
     if (rows <= 0 || rows > 0x7FFFFFFFll || rounds < 0 || n <= 0 || !std::isfinite(lr)) return BMGD_ERR_ARG;
     if (rounds == 0) return BMGD_OK;
     if (n > rows) n = (int)rows;
-    if (h->cfg.loss == BMGD_LOSS_SOFTMAX) {
-        bmgdk::SoftmaxLaunchInfo info{};
-        EventPair ep{};
-        const bool timing = (h->cfg.flags & BMGD_FLAG_TIMING) != 0;
-        if (timing) {
-            int rc = take_events(h, &ep);
-            if (rc != BMGD_OK) return rc;
-            BMGD_CUDA(h, cudaEventRecord(ep.a, h->compute));
-        }
-        int rc = bmgdk::softmax_run(dx, dy, rows, h->cfg.p, h->cfg.C, h->base + h->lay.theta,
-                                   h->base + h->lay.softmax_scratch, reinterpret_cast<int*>(h->base + h->lay.status),
-                                   rounds, n, lr, seed, (h->cfg.flags & BMGD_FLAG_FIXED_PARTITION) ? 1 : 0,
-                                   h->timeout_ns, h->cfg.cluster_size, h->cfg.threads_per_cta,
-                                   (h->cfg.flags & BMGD_FLAG_SOFTMAX_CUDA_CORES) ? 1 : 0,
-                                   h->sm_count, h->smem_optin, h->compute, &info);
-        if (rc != BMGD_OK) {
-            if (info.cuda_error) h->last_cuda = info.cuda_error;
-            if (timing) h->event_pool.push_back(ep);
-            return rc;
-        }
-        if (timing) {
-            BMGD_CUDA(h, cudaEventRecord(ep.b, h->compute));
-            h->kernel_events.push_back(ep);
-        }
-        const int64_t M = (rows + n - 1) / n;
-        h->stats.launches += info.launches;
-        h->stats.steps += (int64_t)rounds * M;
-        h->stats.sample_grads += (int64_t)rounds * rows;
-        h->stats.grid_ctas = info.grid_ctas;
-        h->stats.cluster_size = info.cluster_size;
-        h->stats.ctas_per_chain = info.grid_ctas;
-        h->stats.threads_per_cta = info.threads;
-        h->stats.pipeline_depth = info.depth;
-        h->stats.smem_bytes = info.smem;
-        h->stats.chains_in_flight = 1;
-        return BMGD_OK;
-    }
+    if (h->cfg.loss == BMGD_LOSS_SOFTMAX) return run_softmax(h, dx, dy, rows, rounds, n, lr, seed, false);
     return run_glm(h, dx, dy, rows, rounds, n, lr, seed);
 }
 
@@ -1070,12 +1073,12 @@ int bmgd_gather_buffer(const void* host_x, const void* host_y, int64_t N, int64_
 
 int bmgd_debug_null_rounds(bmgd_t* h, int64_t rows, int32_t rounds, int32_t batch_size) {
     if (!h) return BMGD_ERR_ARG;
-    if (h->cfg.loss == BMGD_LOSS_SOFTMAX) return BMGD_ERR_UNIMPLEMENTED;
     if (rows <= 0 || rows > 0x7FFFFFFFll || rounds < 0 || batch_size <= 0) return BMGD_ERR_ARG;
     if (rounds == 0) return BMGD_OK;
     DeviceGuard guard(h->device);
     if (!guard.ok) return cuda_fail(h, cudaErrorInvalidDevice);
     const int n = batch_size > rows ? (int)rows : batch_size;
+    if (h->cfg.loss == BMGD_LOSS_SOFTMAX) return run_softmax(h, h->base, h->base, rows, rounds, n, 0.0, 0, true);
     // the probe reads no rows; the workspace base stands in for an aligned buffer address
     return run_glm(h, h->base, h->base, rows, rounds, n, 0.0, 0, true);
 }

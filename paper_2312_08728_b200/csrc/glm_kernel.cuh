@@ -175,6 +175,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// the same without suspending the thread: false at once if the phase has not completed
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 // generic-proxy writes to shared memory become ordered with bulk copies into, and tensor-core reads of, the same bytes
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -512,7 +519,9 @@ __device__ __forceinline__ void rows_step(const unsigned char* rowp, int row_str
 __device__ __forceinline__ void bounded_mbar_wait(uint32_t bar, uint32_t parity, bool& aborted, const GlmParams& P) {
     unsigned long long t0 = 0;
     uint32_t spins = 0;
-    while (!aborted && !mbar_try_wait(bar, parity)) {
+    // try_wait suspends the thread in hardware for a while before it answers false; with no budget at all (mask 0) the
+    // wait has to give up at its first look, so it asks without suspending
+    while (!aborted && !(P.mbar_mask ? mbar_try_wait(bar, parity) : mbar_test_wait(bar, parity))) {
         if ((++spins & P.mbar_mask) == 0u) wait_slow_path(t0, aborted, P);
     }
 }

@@ -50,12 +50,14 @@ PHASES_ONE = [("wait for 1st stage", 0, 10), ("sweep", 0, 1), ("cta-sum", 1, 2),
               ("reload", 9, 7)]
 PHASES_MULTI = [("wait for 1st stage", 0, 10), ("sweep", 0, 1), ("cta-sum", 1, 2), ("col-sum", 2, 3), ("rs-push", 3, 4), ("rs-poll+l2-store", 4, 12),
                 ("l2-poll+push", 12, 5), ("totals", 5, 6), ("update", 6, 9), ("reload", 9, 7)]
+PHASES_SOFTMAX = [("wait for rows", 0, 1), ("forward + read-out", 1, 2), ("logits exchange", 2, 3), ("softmax + R push", 3, 4),
+                  ("R arrival", 4, 5), ("backward + read-out", 5, 6), ("update + barrier", 6, 7)]
 PRODUCER = [("shuffle", 0, 1), ("slot+copies A", 1, 3), ("arrive A", 3, 4), ("slot+copies+arrive B", 4, 6)]
 
 
 def trace_workload(L, spec):
     name, _, opts = spec.partition(":")
-    kw, null, chains, rounds = {}, False, 0, 1
+    kw, shape, null, chains, rounds = {}, {}, False, 0, 1
     for o in filter(None, opts.split(",")):
         if o == "null":
             null = True
@@ -65,9 +67,13 @@ def trace_workload(L, spec):
             chains = int(v)
         elif k == "rounds":
             rounds = int(v)
+        elif k in ("p", "n", "N", "K", "C"):  # another shape of the same workload
+            shape[k] = int(v)
         else:
             kw[k] = int(v)
     w = inputs.WORKLOADS[name]
+    if shape:
+        w = w.scaled(**shape)
     if chains:
         w = w.scaled(Rc=chains)
     x, y = inputs.make_buffer(w, 0)
@@ -89,9 +95,12 @@ def trace_workload(L, spec):
           f"{st['threads_per_cta']} threads, ring {st['pipeline_depth']} x {st['subpasses_per_stage']} sub-passes")
     per_blk_step = np.median(t[:nblk, 9:t.shape[1] - 4, 0] - t[:nblk, 8:t.shape[1] - 5, 0], axis=1)
     print(f"   step: {int(per_blk_step[0])} cycles in CTA 0 (min {int(per_blk_step.min())}, max {int(per_blk_step.max())} over CTAs)")
-    for label, a, b in (PHASES_MULTI if multi else PHASES_ONE):
+    softmax = w.loss == inputs.LOSS_SOFTMAX
+    for label, a, b in (PHASES_SOFTMAX if softmax else PHASES_MULTI if multi else PHASES_ONE):
         d = np.median(t[:nblk, steps, b] - t[:nblk, steps, a], axis=1)
         print(f"   {label:18s} {int(d[0]):6d}   (CTAs: min {int(d.min()):6d}  median {int(np.median(d)):6d}  max {int(d.max()):6d})")
+    if softmax:
+        return
     pt = read_stamps(L, 1)
     for label, a, b in PRODUCER:
         d = np.median(pt[:nblk, steps, b] - pt[:nblk, steps, a], axis=1)

@@ -256,7 +256,8 @@ def test_a_wait_that_runs_out_is_reported_and_the_handle_stays_usable():
 @pytest.mark.parametrize("shape", [
     dict(cluster_size=4, ctas_per_chain=4),    # packets inside one cluster
     dict(cluster_size=2, ctas_per_chain=8),    # packets between clusters too
-])  # (a lone CTA waits only on the ring's mbarriers, whose try_wait suspends in hardware and rarely fails twice)
+    dict(cluster_size=1, ctas_per_chain=1),    # only the ring's mbarriers to wait on
+])
 def test_a_step_kernel_wait_that_runs_out_ends_the_launch_and_the_handle_stays_usable(shape):
     """The step kernel's own waits with a budget of a nanosecond: the first wait that does not succeed at its first
     look gives up, every CTA leaves its loops (no copy left in flight, theta not written back), the next
