@@ -411,7 +411,7 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
                     const int half = warp >> 2;
                     if ((tid & 127) == 0) {  // threads 0 and 128 issue one half each
                         if constexpr (!NULLSTEP) {
-                            fence_async_proxy();
+                            // (the rows and the bf16 copy of W were made visible to the tensor core by their writers)
                             tc_fence_after();
                             const uint32_t idesc = tc_idesc(128, kSmxClasses, false);
                             const uint32_t xa = smem_u32(xbuf[b]), wb = smem_u32(wt);

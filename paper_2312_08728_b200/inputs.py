@@ -110,6 +110,28 @@ WORKLOADS = {
 }
 
 
+def _simulation_grid():
+    """The rest of the paper's linear simulation (Section 4.1), same data design as `sim41`.
+
+    First experiment: buffers of 10,000, mini-batches of 1,000, T in {1, 5, 10} at a fixed product alpha T (0.01 here;
+    T = 1 is plain MGD).  Second experiment: T = 5, n in {250, 500, 1000}, K in {2, 5} buffers, 30 passes, with the
+    constant rate alpha = 0.005 (`a`) or alpha = 1/(T K M) (`b`), M = N0 / n mini-batches per buffer."""
+    base = WORKLOADS["sim41"]
+    out = {}
+    for T in (1, 10):
+        out[f"sim41-T{T}"] = dataclasses.replace(base, name=f"sim41-T{T}", T=T, lr=0.01 / T)
+    for K in (2, 5):
+        for n in (250, 500, 1000):
+            M = (base.N // K) // n
+            out[f"sim41-K{K}-n{n}-a"] = dataclasses.replace(base, name=f"sim41-K{K}-n{n}-a", K=K, n=n, T=5, lr=0.005, epochs=30)
+            out[f"sim41-K{K}-n{n}-b"] = dataclasses.replace(base, name=f"sim41-K{K}-n{n}-b", K=K, n=n, T=5,
+                                                            lr=1.0 / (5 * K * M), epochs=30)
+    return out
+
+
+WORKLOADS.update(_simulation_grid())
+
+
 def buffer_seed(base_seed: int, epoch: int, k: int, K: int) -> int:
     """64-bit shuffle seed handed to the call that processes buffer k of pass `epoch`."""
     return (int(base_seed) + epoch * K + k) & 0xFFFFFFFFFFFFFFFF
