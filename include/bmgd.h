@@ -73,7 +73,7 @@ typedef struct bmgd_config {
     int32_t loss;             /* BMGD_LOSS_* */
     int32_t dtype;            /* BMGD_F64 / BMGD_F32 / BMGD_BF16X_F32W */
     int32_t C;                /* classes, softmax only (>= 2); otherwise 1 */
-    int32_t Rc;               /* replicate chains: independent theta's, distinct shuffles, same buffer */
+    int32_t Rc;               /* replicate chains: independent theta's, distinct shuffles, same buffer (any loss) */
     int32_t device;           /* CUDA device ordinal; -1 = the calling thread's current device */
     uint32_t flags;           /* BMGD_FLAG_* */
     void*   workspace;        /* dev memory, 256-byte aligned, owned by the caller and kept alive until
@@ -85,7 +85,7 @@ typedef struct bmgd_config {
      * (a multiple of cluster_size); the rows of a mini-batch are split among them. */
     int32_t cluster_size;     /* CTAs per thread-block cluster: 1, 2, 4, 8 or 16 */
     int32_t ctas_per_chain;
-    int32_t threads_per_cta;  /* threads that compute: a multiple of 32 from 256 to 512 (softmax: 256, 512 or 1024) */
+    int32_t threads_per_cta;  /* linear/logistic: threads that compute, a multiple of 32 from 256 to 512 (softmax: fixed) */
     int32_t pipeline_depth;   /* row-prefetch stages held in shared memory: 2 to 8 */
     int32_t subpasses_per_stage; /* a stage holds this many sweeps of the CTA over its rows: 1, 2, 4, ... 32 */
     int32_t producer_warps;   /* linear/logistic: extra warps per CTA that only evaluate the shuffle and fetch rows: 1 to 8 */
@@ -149,6 +149,8 @@ int bmgd_load_buffer(bmgd_t* h, const void* host_x, const void* host_y, int64_t 
  * may be shorter and is averaged by its own size), learning rate lr, for every chain.  Round t
  * of chain c uses the partition keyed by (seed, c, t).  Asynchronous on the compute stream;
  * waits on-stream for the slot's copy.  theta is updated in place on the device.
+ * Softmax handles (bf16 rows, fp32 W): at most 16 classes, batch_size at most 256, p a multiple of 8 up to 3072;
+ * other shapes return BMGD_ERR_UNIMPLEMENTED.
  */
 int bmgd_run_rounds(bmgd_t* h, int32_t slot, int32_t rounds, int32_t batch_size, double lr,
                     uint64_t seed);
@@ -178,14 +180,17 @@ int bmgd_run_rounds_resident(bmgd_t* h, const void* dev_x, const void* dev_y, in
  * defaults) for the least-squares and logistic losses in BMGD_F32 or BMGD_F64, on the calling
  * thread's current device, ordered on `stream` (a cudaStream_t; NULL = the legacy default
  * stream).  dev_theta [Rc][p] is the caller's: it is read as the starting value and holds the
- * result.  The call returns after the kernel has finished.
+ * result.  The call returns after the kernel has finished: it synchronises `stream` itself (that is how
+ * it reads the kernel's status words back), so it cannot run inside a stream capture.  Device-side
+ * waits are bounded by a fixed 2000 ms (a handle's timeout_ms has no counterpart here); a wait that gives
+ * up returns BMGD_ERR_TIMEOUT from this very call.
  *
  * Limits and sharing: p must not exceed BMGD_NOALLOC_MAX_P, else BMGD_ERR_CAPACITY is returned
  * and nothing runs.  All calls on one GPU, from any thread or stream, use the same array; it
  * keeps the contents of the previous call, so each call first clears the part it uses.  Two
  * calls that overlap in time on one GPU would race on it: issue them one after the other.
- * The first call on each device looks up the array's device address; make that first call
- * outside any stream capture.
+ * The first call on each device also looks up the array's device address (cudaGetSymbolAddress, once
+ * per device, with that device current).
  */
 #define BMGD_NOALLOC_MAX_P 256
 #define BMGD_NOALLOC_SCRATCH_BYTES (256 + 2 * 160 * BMGD_NOALLOC_MAX_P * 2 * 8)
@@ -261,7 +266,7 @@ int bmgd_gather_buffer(const void* host_x, const void* host_y, int64_t N, int64_
                        int32_t K, uint64_t seed, uint32_t pass, int32_t k, void* stage_x, void* stage_y,
                        int32_t threads, int64_t* rows_out);
 
-/* Latency probe of the computation step (linear and logistic handles): launch, on the compute stream, the step
+/* Latency probe of the computation step: launch, on the compute stream, the step
  * kernel's own synchronisation structure for a buffer of `rows` rows, `rounds` rounds and mini-batches of
  * batch_size rows, in the launch shape bmgd_run_rounds would choose, with every ring hand-over, barrier, packet
  * exchange between CTAs and update of a step, but without fetching or multiplying a single row (the gradient is
