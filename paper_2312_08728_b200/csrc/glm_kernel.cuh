@@ -667,7 +667,8 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                     cp_async_fill<(int)sizeof(T)>(stage_base + (uint32_t)(plan.stage_y_off + (s0 + lane) * (int)sizeof(T)),
                                                   yb + (have ? rows : 0u), have);
                 }
-                return (uint32_t)__popc(__ballot_sync(0xFFFFFFFFu, mine));
+                // gathers issued for this batch: one per four slots that exist (the same in every lane: no vote needed)
+                return (uint32_t)min(8, (left + 3) >> 2);
             } else if constexpr (CB == 16) {
                 const bool have = lane < left && rows != kNoRow;
                 const uint32_t dst = stage_base + (uint32_t)((s0 + lane) * pitch);
@@ -730,7 +731,8 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
             if (two && ++slot == D) { slot = 0; empty_parity ^= 1u; }
             const uint32_t baseA = ring_base + (uint32_t)(slotA * stage_bytes), baseB = ring_base + (uint32_t)(slotB * stage_bytes);
             const int b0 = (int)rot;  // this producer's first batch in this pair of stages
-            rot = (rot + (uint32_t)NPW - rot_step) % (uint32_t)NPW;
+            rot += (uint32_t)NPW - rot_step;  // below 2 * NPW
+            if (rot >= (uint32_t)NPW) rot -= (uint32_t)NPW;
 
             // the shuffle of both stages first (it needs no ring slot), then the copies of A, then those of B
             uint32_t rowsA[kMaxBatchesPerProducer], rowsB[kMaxBatchesPerProducer];
