@@ -149,8 +149,8 @@ int bmgd_load_buffer(bmgd_t* h, const void* host_x, const void* host_y, int64_t 
  * may be shorter and is averaged by its own size), learning rate lr, for every chain.  Round t
  * of chain c uses the partition keyed by (seed, c, t).  Asynchronous on the compute stream;
  * waits on-stream for the slot's copy.  theta is updated in place on the device.
- * Softmax handles (bf16 rows, fp32 W): at most 16 classes, batch_size at most 256, p a multiple of 8 up to 3072;
- * other shapes return BMGD_ERR_UNIMPLEMENTED.
+ * Softmax handles (bf16 rows, fp32 W): at most 16 classes, p a multiple of 8 up to 3072 (any batch_size: a
+ * mini-batch of more than 256 rows is taken in tiles of 256); other shapes return BMGD_ERR_UNIMPLEMENTED.
  */
 int bmgd_run_rounds(bmgd_t* h, int32_t slot, int32_t rounds, int32_t batch_size, double lr,
                     uint64_t seed);

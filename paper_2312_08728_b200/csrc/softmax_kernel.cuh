@@ -59,6 +59,7 @@ struct SoftmaxParams {
     double scale_full, scale_last;
     uint32_t N0, n, M;
     int T, p, C, S, NP, Rc, nclusters;
+    int ntile;          // tiles of 256 row slots per mini-batch
     uint32_t chain0;
     int fixed_partition;
     uint32_t mbar_mask;
@@ -223,7 +224,11 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
     const FeistelDomain dom = make_domain(N0);
     WaitCtx wc{P.status, P.timeout_ns, P.mbar_mask, false};
     const int nch = (cluster < P.Rc) ? (P.Rc - cluster + P.nclusters - 1) / P.nclusters : 0;
-    const uint32_t steps_per_chain = (uint32_t)P.T * M;
+    // A mini-batch of more than 256 rows is taken in `ntile` tiles of 256 row slots: each tile goes through the gather,
+    // the forward contraction, the two exchanges and the backward contraction on its own (the backward one adds into
+    // the same accumulators); W is updated after the last tile.  "step" below counts tiles.
+    const uint32_t ntile = (uint32_t)P.ntile;
+    const uint32_t steps_per_chain = (uint32_t)P.T * M * ntile;
     const uint32_t total_steps = (uint32_t)nch * steps_per_chain;
     const int zchunks = (C + 3) >> 2;       // 16-byte pieces of a row's logits that carry real classes
     const int ntiles = NP > 2 ? 2 : 1;      // backward tiles of 128 predictors (tile 1: predictors 64..191)
@@ -260,10 +265,12 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
         cluster_wait_acquire();
     }
 
-    auto step_rows = [&](uint32_t step, uint32_t& lo, uint32_t& nm) {
-        const uint32_t m = (step % steps_per_chain) % M;
-        lo = m * n;
-        nm = min(n, N0 - lo);
+    auto step_rows = [&](uint32_t step, uint32_t& lo, uint32_t& nm) {  // rows [lo, lo + nm) of the round's order: this tile's
+        const uint32_t in_chain = step % steps_per_chain;
+        const uint32_t m = (in_chain / ntile) % M, tau = in_chain % ntile;
+        const uint32_t batch = min(n, N0 - m * n);
+        lo = m * n + tau * (uint32_t)kSmxRows;
+        nm = batch > tau * (uint32_t)kSmxRows ? min((uint32_t)kSmxRows, batch - tau * (uint32_t)kSmxRows) : 0u;
     };
 
     if (warp >= kSmxCompute / 32) {
@@ -283,7 +290,7 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
         for (uint32_t step = 0; step < total_steps; ++step) {
             const int b = (int)(step & 1u);
             const uint32_t ci = step / steps_per_chain;
-            const uint32_t t = P.fixed_partition ? 0u : (step % steps_per_chain) / M;
+            const uint32_t t = P.fixed_partition ? 0u : (step % steps_per_chain) / (M * ntile);
             if (ci != rk_chain || t != rk_round) {
                 rk = round_keys(P.seed, P.chain0 + (uint32_t)(cluster + (int)ci * P.nclusters), t);
                 rk_chain = ci; rk_round = t;
@@ -385,13 +392,18 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
             write_wt();
             named_sync(1, kSmxCompute);
 
-            uint32_t m = 0;  // mini-batch of the round (kept by counting: no division at the head of a step)
+            uint32_t m = 0, tau = 0;  // mini-batch of the round and tile of the mini-batch (kept by counting: no division here)
+            float gr_cc[kSmxClasses];  // CUDA-core path: the gradient row of this thread's predictor, summed over the tiles
+#pragma unroll
+            for (int c = 0; c < kSmxClasses; ++c) gr_cc[c] = 0.f;
             for (uint32_t s_in = 0; s_in < steps_per_chain; ++s_in, ++step) {
                 const int b = (int)(step & 1u);
-                const uint32_t par = step & 1u;           // phase parity of the once-per-step barriers
+                const uint32_t par = step & 1u;           // phase parity of the once-per-tile barriers
                 const uint32_t xpar = (step >> 1) & 1u;   // and of the per-buffer ones
-                const uint32_t lo = m * n, nm = min(n, N0 - lo);
-                if (++m == M) m = 0;
+                const uint32_t batch = min(n, N0 - m * n);  // rows of the mini-batch
+                const uint32_t nm = batch > tau * (uint32_t)kSmxRows ? min((uint32_t)kSmxRows, batch - tau * (uint32_t)kSmxRows) : 0u;
+                const bool first_tile = tau == 0, last_tile = tau + 1 == ntile;
+                if (++tau == ntile) { tau = 0; if (++m == M) m = 0; }
 #ifdef BMGD_TRACE
                 const uint32_t step_count = step;
 #endif
@@ -532,7 +544,7 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
                                 const uint32_t b_addr = rb + (uint32_t)((ks >> 2) * kSmxClasses * 128 + (ks & 3) * 32);
                                 tc_mma_bf16(tmem_base + (uint32_t)(((2 + tile) * kSmxAcc + (ks % kSmxAcc)) * kSmxClasses),
                                             tc_smem_desc(a_addr, kSmxRows * 128, 1024), tc_smem_desc(b_addr, 16, 1024), idesc,
-                                            ks >= kSmxAcc ? 1u : 0u);
+                                            (ks >= kSmxAcc || !first_tile) ? 1u : 0u);
                             }
                             tc_commit(gbar + (uint32_t)(tile * 8));
                         } else {
@@ -541,7 +553,7 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
                     }
                     if (tile < ntiles) {
                         mbar_wait(gbar + (uint32_t)(tile * 8), par, wc);
-                        if constexpr (!NULLSTEP) {
+                        if (!NULLSTEP && last_tile) {
                             tc_fence_after();
                             if (tid < 128) tc_load_sum(tmem_base + ((uint32_t)((warp & 3) * 32) << 16), (uint32_t)(2 * kSmxAcc * kSmxClasses), gr);
                             else if (tid >= 192) tc_load_sum(tmem_base + ((uint32_t)((warp & 3) * 32) << 16), (uint32_t)(3 * kSmxAcc * kSmxClasses), gr);
@@ -558,8 +570,12 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
                                 xbuf[b] + smx_chunk_off(row, my_f >> 3, kSmxRows) + (my_f & 7) * 2));
                             const __nv_bfloat16* rr = reinterpret_cast<const __nv_bfloat16*>(rbuf + row * kSmxClasses * 2);
 #pragma unroll
-                            for (int c = 0; c < kSmxClasses; ++c) gr[c] = fmaf(xf, __bfloat162float(rr[c]), gr[c]);
+                            for (int c = 0; c < kSmxClasses; ++c) gr_cc[c] = fmaf(xf, __bfloat162float(rr[c]), gr_cc[c]);
                         }
+                    }
+                    if (last_tile) {
+#pragma unroll
+                        for (int c = 0; c < kSmxClasses; ++c) { gr[c] = gr_cc[c]; gr_cc[c] = 0.f; }
                     }
                     named_sync(3, kSmxCompute);  // every thread has read the rows and the residuals
                     if (tid == 0) mbar_arrive(xempty + (uint32_t)(b * 8));
@@ -567,13 +583,17 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
                 BMGD_STAMP(6);
 
                 // ---- update of W_slice and of its bf16 copy
-                const float scale = (float)((nm == n) ? P.scale_full : P.scale_last);
-                if (owns_w) {
+                if (last_tile) {
+                    const float scale = (float)((batch == n) ? P.scale_full : P.scale_last);
+                    if (owns_w) {
 #pragma unroll
-                    for (int c = 0; c < kSmxClasses; ++c) w[c] = fmaf(-scale, gr[c], w[c]);
+                        for (int c = 0; c < kSmxClasses; ++c) w[c] = fmaf(-scale, gr[c], w[c]);
+                    }
+                    write_wt();
                 }
-                write_wt();
-                named_sync(1, kSmxCompute);  // the bf16 copy is complete before the next forward contraction reads it
+                // every thread is past this tile's contractions (the residual buffer and the tensor-memory tiles may be
+                // reused) and, after the last tile, the bf16 copy is complete before the next forward contraction reads it
+                named_sync(1, kSmxCompute);
                 BMGD_STAMP(7);
                 if (stop) goto compute_done;  // the same decision in every compute thread; W is not written back
             }
@@ -600,15 +620,15 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
 
 // ---------------------------------------------------------------- host side
 
-// Runs `rounds` rounds over the buffer on `stream` for Rc chains.  Shapes this kernel covers: C <= 16, batch_size <= 256,
-// p a multiple of 8 (rows are 16-byte multiples) up to 16 * 192; the predictors are spread over the smallest cluster of
+// Runs `rounds` rounds over the buffer on `stream` for Rc chains.  Shapes this kernel covers: C <= 16, any batch size
+// (taken in tiles of 256 rows), p a multiple of 8 (rows are 16-byte multiples) up to 16 * 192; the predictors are spread over the smallest cluster of
 // S in {1, 2, 4, 8, 16} CTAs whose slices of 64, 128 or 192 predictors hold them.  Returns a bmgd_status value.
 inline int softmax_run(const void* dx, const void* dy, int64_t rows, int p, int C, int Rc, uint32_t chain0, void* W, int* status,
                        int rounds, int n, double lr, unsigned long long seed, int fixed, unsigned long long timeout_ns,
                        int cluster_size, int use_cuda_cores, int null_step, int smem_optin, cudaStream_t stream,
                        SoftmaxLaunchInfo* info) {
     *info = SoftmaxLaunchInfo{};
-    if (C > kSmxClasses || n > kSmxRows || p % 8 != 0) return -8;
+    if (C > kSmxClasses || p % 8 != 0) return -8;
     int S = 0, NP = 0;
     for (int s = 1; s <= 16 && !S; s <<= 1) {
         if (cluster_size && s != cluster_size) continue;
@@ -650,7 +670,8 @@ inline int softmax_run(const void* dx, const void* dy, int64_t rows, int p, int 
     if (nclusters < 1) return -7;
     nclusters = nclusters < Rc ? nclusters : Rc;  // clusters are independent: no need for all of them to be resident at once
     const int chains_per_cluster = (Rc + nclusters - 1) / nclusters;
-    if ((uint64_t)chains_per_cluster * (uint64_t)rounds * M >= 0xFFFFFFF0ull) return -1;
+    const int ntile = (n + kSmxRows - 1) / kSmxRows;
+    if ((uint64_t)chains_per_cluster * (uint64_t)rounds * M * (uint64_t)ntile >= 0xFFFFFFF0ull) return -1;
     lc.gridDim = dim3((unsigned)(S * nclusters), 1, 1);
 
     SoftmaxParams P{};
@@ -659,7 +680,7 @@ inline int softmax_run(const void* dx, const void* dy, int64_t rows, int p, int 
     P.scale_full = lr / (double)n;
     P.scale_last = lr / (double)(rows - (int64_t)(M - 1) * n);
     P.N0 = (uint32_t)rows; P.n = (uint32_t)n; P.M = M; P.T = rounds; P.p = p; P.C = C; P.S = S; P.NP = NP;
-    P.Rc = Rc; P.nclusters = nclusters; P.chain0 = chain0;
+    P.Rc = Rc; P.nclusters = nclusters; P.chain0 = chain0; P.ntile = ntile;
     P.fixed_partition = fixed;
     const bool tiny = timeout_ns < 1000ull;  // below a microsecond: no budget at all, every failed look gives up
     if (tiny) P.timeout_ns = 0;

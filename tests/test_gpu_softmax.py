@@ -92,6 +92,14 @@ def test_predictor_counts_that_do_not_fill_the_last_panel(p):
     check(job(p, N=600, T=1), CUDA_CORES)
 
 
+@pytest.mark.parametrize("p,N,n", [(384, 1_500, 300), (1024, 2_100, 512), (3072, 1_300, 1_000), (128, 2_000, 2_000)])
+def test_mini_batches_larger_than_one_tile(p, N, n):
+    """More than 256 rows per mini-batch: the step takes them in tiles of 256 row slots (the last tile and the last
+    mini-batch ragged, one case with a single full-batch step per round), the gradient summed over the tiles before W moves."""
+    check(job(p, N=N, n=n, T=2), 0)
+    check(job(p, N=N, n=n, T=1), CUDA_CORES)
+
+
 def test_replicate_chains_one_cluster_per_chain():
     """Four chains with their own W and their own partitions over one buffer, one cluster of CTAs each, in one launch;
     and more chains than clusters fit (a cluster then takes its chains one after the other).  Every chain against
@@ -145,7 +153,7 @@ def test_a_softmax_wait_that_runs_out_is_reported_and_the_handle_stays_usable():
 
 def test_unsupported_shapes_are_refused_not_miscomputed():
     from paper_2312_08728_b200.binding import BmgdError, ERR_UNIMPLEMENTED
-    for w in (job(100), job(384, n=300), job(3080)):
+    for w in (job(100), job(384, C=17), job(3080)):
         with pytest.raises(BmgdError) as e:
             gpu_job(w, buffers_of(w), mode="resident")
         assert e.value.status == ERR_UNIMPLEMENTED
