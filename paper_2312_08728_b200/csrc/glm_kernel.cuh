@@ -517,6 +517,7 @@ __device__ __forceinline__ void rows_step(const unsigned char* rowp, int row_str
 
 // Waits for a phase of an mbarrier in this CTA's shared memory with the kernel's bounded-wait protocol.
 __device__ __forceinline__ void bounded_mbar_wait(uint32_t bar, uint32_t parity, bool& aborted, const GlmParams& P) {
+    if (mbar_test_wait(bar, parity)) return;  // the usual case where the ring runs ahead: the phase is long complete
     unsigned long long t0 = 0;
     uint32_t spins = 0;
     // try_wait suspends the thread in hardware for a while before it answers false; with no budget at all (mask 0) the
@@ -884,6 +885,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                     int sp_left = sp_full;
                     if (!full_batch) sp_left = (sh.cnt > warp_first) ? (int)((sh.cnt - warp_first - 1u) / (uint32_t)spp) + 1 : 0;
                     for (int sidx = 0; sidx < passes; ++sidx) {
+                        if (sidx == 0) BMGD_STAMP(11);
                         bounded_mbar_wait(full_bars + (uint32_t)(cs_slot * 8), cs_phase, aborted, P);
                         __syncwarp();
                         if (sidx == 0) BMGD_STAMP(10);
@@ -904,6 +906,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                             }
                         }
                         if (nsub) row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, yp, th, gacc);
+                        if (sidx == 0) BMGD_STAMP(13);
                         __syncwarp();  // every lane has its values in registers: the slot may be refilled
                         if (lane == 0) mbar_arrive(empty_bars + (uint32_t)(cs_slot * 8));
                         if (++cs_slot == D) { cs_slot = 0; cs_phase ^= 1u; }

@@ -116,7 +116,10 @@ struct WaitCtx {
     uint32_t mask;
     bool aborted;
 };
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, WaitCtx& w) {
+// `likely_done`: the phase has usually completed long before (a buffer filled a step ahead): ask once without suspending
+// the thread first, which answers faster than try_wait does even on a completed phase.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, WaitCtx& w, bool likely_done = false) {
+    if (likely_done && mbar_test_wait(bar, parity)) return;
     unsigned long long t0 = 0;
     uint32_t spins = 0;
     // (with no budget at all, mask 0, the wait asks without suspending the thread: it gives up at its first look)
@@ -301,7 +304,7 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
             uint32_t r = 0xFFFFFFFFu;
             if (!NULLSTEP && lane < kSlots && (uint32_t)slot < nm) r = perm_index(lo + (uint32_t)slot, dom, rk);
             // the buffer's last reader (the backward contraction two steps ago) must have finished
-            mbar_wait(xempty + (uint32_t)(b * 8), ((step >> 1) & 1u) ^ 1u, wc);
+            mbar_wait(xempty + (uint32_t)(b * 8), ((step >> 1) & 1u) ^ 1u, wc, true);
             wc.aborted = __any_sync(0xFFFFFFFFu, wc.aborted);
             if (wc.aborted) break;
             if constexpr (!NULLSTEP) {
@@ -412,7 +415,7 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
                     if (S > 1) { mbar_arrive_expect_tx(zbar, z_expect); mbar_arrive_expect_tx(rbar, r_expect); }
                     else { mbar_arrive(zbar); mbar_arrive(rbar); }
                 }
-                mbar_wait(xfull + (uint32_t)(b * 8), xpar, wc);  // this step's rows (gathered during the previous step)
+                mbar_wait(xfull + (uint32_t)(b * 8), xpar, wc, true);  // this step's rows (gathered during the previous step)
                 BMGD_STAMP(1);
 
                 // ---- forward: partial logits of row slot `tid` over this CTA's predictors

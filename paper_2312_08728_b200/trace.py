@@ -46,9 +46,9 @@ def read_stamps(L, which=0):
 
 
 # (name, from phase, to phase) for one cluster per chain and for several
-PHASES_ONE = [("wait for 1st stage", 0, 10), ("sweep", 0, 1), ("cta-sum", 1, 2), ("col-sum", 2, 3), ("push", 3, 8), ("poll", 8, 4), ("update", 6, 9),
+PHASES_ONE = [("step head", 0, 11), ("wait for 1st stage", 11, 10), ("1st stage's rows", 10, 13), ("sweep", 0, 1), ("cta-sum", 1, 2), ("col-sum", 2, 3), ("push", 3, 8), ("poll", 8, 4), ("update", 6, 9),
               ("reload", 9, 7)]
-PHASES_MULTI = [("wait for 1st stage", 0, 10), ("sweep", 0, 1), ("cta-sum", 1, 2), ("col-sum", 2, 3), ("rs-push", 3, 4), ("rs-poll+l2-store", 4, 12),
+PHASES_MULTI = [("step head", 0, 11), ("wait for 1st stage", 11, 10), ("1st stage's rows", 10, 13), ("sweep", 0, 1), ("cta-sum", 1, 2), ("col-sum", 2, 3), ("rs-push", 3, 4), ("rs-poll+l2-store", 4, 12),
                 ("l2-poll+push", 12, 5), ("totals", 5, 6), ("update", 6, 9), ("reload", 9, 7)]
 PHASES_SOFTMAX = [("wait for rows", 0, 1), ("forward + read-out", 1, 2), ("logits exchange", 2, 3), ("softmax + R push", 3, 4),
                   ("R arrival", 4, 5), ("backward + read-out", 5, 6), ("update + barrier", 6, 7)]
