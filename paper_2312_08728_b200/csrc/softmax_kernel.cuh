@@ -411,7 +411,7 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
                 const uint32_t step_count = step;
 #endif
                 BMGD_STAMP(0);
-                if (tid == 0) {  // this step's incoming bytes (they may start to arrive before this line runs)
+                if (tid == 64) {  // this step's incoming bytes (they may start to arrive before this line runs); a thread of a warp that issues no contraction
                     if (S > 1) { mbar_arrive_expect_tx(zbar, z_expect); mbar_arrive_expect_tx(rbar, r_expect); }
                     else { mbar_arrive(zbar); mbar_arrive(rbar); }
                 }
