@@ -11,10 +11,8 @@ CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libbmgd.so")
 TRACE_LIB_PATH = os.path.join(_PKG, "libbmgd_trace.so")  # the same sources with -DBMGD_TRACE (phase clock stamps)
 
-NVCC_FLAGS = [
-    "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-shared", "-Xcompiler", "-fPIC",
-]
+NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC"]
+BUILD_DIR = os.path.join(_PKG, "_build")  # object files (kept out of the history)
 
 
 def _sources():
@@ -51,10 +49,19 @@ def build(force: bool = False, verbose: bool = False, trace: bool = False) -> st
     nvcc = find_nvcc()
     if nvcc is None:
         raise RuntimeError("nvcc not found: cannot build the BMGD CUDA library")
+    # the tables of step kernels are translation units of their own: compile all of them side by side, then link
+    flags = NVCC_FLAGS + (["-DBMGD_TRACE"] if trace else []) + (["-Xptxas", "-v"] if verbose else [])
+    objdir = os.path.join(BUILD_DIR, "trace" if trace else "lib")
+    os.makedirs(objdir, exist_ok=True)
+    jobs = []
+    for src in _sources():
+        obj = os.path.join(objdir, os.path.splitext(os.path.basename(src))[0] + ".o")
+        jobs.append((obj, subprocess.Popen([nvcc] + flags + ["-c", "-o", obj, src], cwd=CSRC)))
+    failed = [obj for obj, proc in jobs if proc.wait() != 0]
+    if failed:
+        raise RuntimeError("nvcc failed for " + ", ".join(os.path.basename(o) for o in failed))
     tmp = out + f".{os.getpid()}.tmp"
-    cmd = ([nvcc] + NVCC_FLAGS + (["-DBMGD_TRACE"] if trace else []) + (["-Xptxas", "-v"] if verbose else [])
-           + ["-o", tmp] + _sources() + ["-lcudart"])
-    subprocess.check_call(cmd, cwd=CSRC)
+    subprocess.check_call([nvcc, "-shared"] + NVCC_FLAGS[:2] + ["-o", tmp] + [obj for obj, _ in jobs] + ["-lcudart"], cwd=CSRC)
     os.replace(tmp, out)
     return out
 

@@ -15,12 +15,15 @@
 #include <thread>
 #include <vector>
 
-#include "glm_kernel.cuh"
+#include "aux_kernels.cuh"
+#include "glm_table.cuh"
 #include "softmax_kernel.cuh"
 
 namespace {
 
+using bmgdk::GlmKernel;
 using bmgdk::GlmParams;
+using bmgdk::GlmVariant;
 
 constexpr int64_t kAlign = 256;
 constexpr int kMaxClustersForExchange = 160;  // upper bound on clusters in one grid (148 SMs)
@@ -203,57 +206,15 @@ int make_row_map(const void* dev_x, int64_t rows, int p, int elem_bytes, int box
 
 // ------------------------------------------------------------------ GLM kernel table
 
-typedef void (*GlmKernel)(const GlmParams, const CUtensorMap);
-
-struct GlmVariant {
-    GlmKernel fn_small;  // compiled for CTAs of up to kGlmSmallCta threads (more registers per thread)
-    GlmKernel fn_large;  // compiled for CTAs of up to kGlmLargeCta threads, or null
-    GlmKernel null_small, null_large;  // the latency probe of the same shape (least-squares tables only)
-    GlmKernel fn(int cta_threads, bool null_step = false) const {
-        const bool large = cta_threads > bmgdk::kGlmSmallCta && fn_large;
-        return null_step ? (large ? null_large : null_small) : (large ? fn_large : fn_small);
-    }
-    int vec, lpr, kch, maxc, maxt;
-    int cap() const { return vec * lpr * kch; }
-    int max_consumer_threads() const { return maxc; }  // warps that compute
-    int max_threads() const { return maxt; }           // consumers plus producers
-};
-
-// The latency probe does not depend on the loss: it is built once, beside the least-squares kernels.
-template <typename T, int VEC, int LPR, int KCH, bool LG, int MAXT>
-constexpr GlmKernel glm_null_kernel() {
-    if constexpr (LG) return nullptr;
-    else return bmgdk::glm_kernel<T, VEC, LPR, KCH, false, MAXT, true>;
-}
-
-template <typename T, bool LG>
-const GlmVariant* glm_variants(bool aligned16, int* count) {
-    constexpr int V = 16 / (int)sizeof(T);
-#define BMGD_VAR(VEC, LPR, KCH) {bmgdk::glm_kernel<T, VEC, LPR, KCH, LG, bmgdk::kGlmSmallCta>, \
-                                 (bmgdk::glm_max_threads<T, VEC, KCH>() != bmgdk::kGlmSmallCta) \
-                                     ? bmgdk::glm_kernel<T, VEC, LPR, KCH, LG, bmgdk::glm_max_threads<T, VEC, KCH>()> : nullptr, \
-                                 glm_null_kernel<T, VEC, LPR, KCH, LG, bmgdk::kGlmSmallCta>(), \
-                                 (bmgdk::glm_max_threads<T, VEC, KCH>() != bmgdk::kGlmSmallCta) \
-                                     ? glm_null_kernel<T, VEC, LPR, KCH, LG, bmgdk::glm_max_threads<T, VEC, KCH>()>() : nullptr, \
-                                 VEC, LPR, KCH, \
-                                 bmgdk::glm_max_consumer_threads<T, VEC, KCH>(), bmgdk::glm_max_threads<T, VEC, KCH>()}
-    // ordered by capacity; among equal capacities the one listed first is the default, the others are reached
-    // through cfg.lanes_per_row
-    static const GlmVariant wide[] = {BMGD_VAR(V, 8, 1), BMGD_VAR(V, 8, 2), BMGD_VAR(V, 4, 4), BMGD_VAR(V, 4, 7),
-                                      BMGD_VAR(V, 8, 4), BMGD_VAR(V, 8, 8), BMGD_VAR(V, 16, 8), BMGD_VAR(V, 32, 8)};
-    static const GlmVariant narrow[] = {BMGD_VAR(1, 32, 1), BMGD_VAR(1, 32, 2), BMGD_VAR(1, 32, 4), BMGD_VAR(1, 32, 8)};
-#undef BMGD_VAR
-    if (aligned16) { *count = 8; return wide; }
-    *count = 4;
-    return narrow;
-}
-
-const GlmVariant* pick_variant(int dtype, int loss, int p, bool aligned16, int lanes_per_row = 0) {
+// null_step: the latency probe of that shape instead of the step kernel (it does not depend on the loss)
+const GlmVariant* pick_variant(int dtype, int loss, int p, bool aligned16, int lanes_per_row = 0, bool null_step = false) {
     int cnt = 0;
     const bool lg = loss == BMGD_LOSS_LOGISTIC;
-    const GlmVariant* v = dtype == BMGD_F64
-        ? (lg ? glm_variants<double, true>(aligned16, &cnt) : glm_variants<double, false>(aligned16, &cnt))
-        : (lg ? glm_variants<float, true>(aligned16, &cnt) : glm_variants<float, false>(aligned16, &cnt));
+    const GlmVariant* v = null_step
+        ? (dtype == BMGD_F64 ? bmgdk::glm_variants_f64_null(aligned16, &cnt) : bmgdk::glm_variants_f32_null(aligned16, &cnt))
+        : dtype == BMGD_F64
+        ? (lg ? bmgdk::glm_variants_f64_logistic(aligned16, &cnt) : bmgdk::glm_variants_f64_linear(aligned16, &cnt))
+        : (lg ? bmgdk::glm_variants_f32_logistic(aligned16, &cnt) : bmgdk::glm_variants_f32_linear(aligned16, &cnt));
     if (lanes_per_row)  // the smallest variant with that many lanes per row, if there is one
         for (int i = 0; i < cnt; ++i)
             if (v[i].cap() >= p && v[i].lpr == lanes_per_row) return &v[i];
@@ -297,7 +258,7 @@ int max_active_clusters(bmgd* h, GlmKernel fn, int S, int threads, int smem, int
     return BMGD_OK;
 }
 
-int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* out, bool null_step = false) {
+int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* out) {
     const bmgd_config& c = h->cfg;
     const int eb = h->tb;
     const int gpw = 32 / var->lpr;
@@ -344,11 +305,16 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
             return BMGD_ERR_UNIMPLEMENTED;
         }
         const int probe_smem = fixed_smem + ring_budget;
-        BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn(L.threads + 32 * L.pwarps, null_step), cudaFuncAttributeMaxDynamicSharedMemorySize, probe_smem));
-        BMGD_CUDA(h, cudaFuncSetAttribute((const void*)var->fn(L.threads + 32 * L.pwarps, null_step), cudaFuncAttributeNonPortableClusterSizeAllowed, S > 8 ? 1 : 0));
+        // whichever flavour the launch takes in the end (that depends on the clusters per chain chosen below), it runs
+        // with these limits; all flavours have the same launch bounds, so one answers for all on residency
+        for (int fl = 0; fl < bmgdk::kGlmFlavours; ++fl) {
+            const void* fn = (const void*)var->fn(L.threads + 32 * L.pwarps, fl);
+            BMGD_CUDA(h, cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, probe_smem));
+            BMGD_CUDA(h, cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, S > 8 ? 1 : 0));
+        }
         max_clusters = h->sm_count;
         if (S > 1) {
-            int rc = max_active_clusters(h, var->fn(L.threads + 32 * L.pwarps, null_step), S, L.threads + 32 * L.pwarps, probe_smem, &max_clusters);
+            int rc = max_active_clusters(h, var->fn(L.threads + 32 * L.pwarps, bmgdk::kGlmAny), S, L.threads + 32 * L.pwarps, probe_smem, &max_clusters);
             if (rc != BMGD_OK) {
                 if (c.cluster_size == 0 && S > 8) { S = 8; continue; }  // clusters of 16 are optional in hardware
                 return rc;
@@ -451,11 +417,11 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
             bool null_step = false) {
     const bmgd_config& c = h->cfg;
     const bool aligned16 = ((int64_t)c.p * h->tb) % 16 == 0 && ((uintptr_t)dx % 16) == 0;
-    const GlmVariant* var = pick_variant(c.dtype, null_step ? BMGD_LOSS_LINEAR : c.loss, c.p, aligned16, c.lanes_per_row);
+    const GlmVariant* var = pick_variant(c.dtype, c.loss, c.p, aligned16, c.lanes_per_row, null_step);
     if (!var) return BMGD_ERR_UNIMPLEMENTED;
     if (((uintptr_t)dx % h->tb) != 0 || ((uintptr_t)dy % h->tb) != 0) return BMGD_ERR_ARG;
     LaunchShape L{};
-    int rc = plan_glm(h, var, rows, n, &L, null_step);
+    int rc = plan_glm(h, var, rows, n, &L);
     if (rc != BMGD_OK) return rc;
 
     const uint32_t M = (uint32_t)((rows + n - 1) / n);
@@ -496,6 +462,9 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
     P.chain0 = (uint32_t)c.first_chain;
     P.fixed_partition = (c.flags & BMGD_FLAG_FIXED_PARTITION) ? 1 : 0;
     set_poll_cadence(&P);
+#ifdef BMGD_TRACE
+    P.trace = bmgdk::trace_buffer(0); P.ptrace = bmgdk::trace_buffer(1);
+#endif
     if ((int64_t)L.nteams * L.cpc > kMaxClustersForExchange) return BMGD_ERR_LAUNCH;
 
     cudaLaunchConfig_t lc{};
@@ -533,7 +502,7 @@ int run_glm(bmgd* h, const void* dx, const void* dy, int64_t rows, int rounds, i
             return rc;
         }
     }
-    cudaError_t e = cudaLaunchKernelEx(&lc, var->fn(L.threads + 32 * L.pwarps, null_step), P, xmap);
+    cudaError_t e = cudaLaunchKernelEx(&lc, var->fn(L.threads + 32 * L.pwarps, bmgdk::glm_flavour(P.opt_kind, P.sched, L.cpc)), P, xmap);
     if (e != cudaSuccess) {
         h->last_cuda = (int)e;
         cudaGetLastError();
@@ -1005,7 +974,7 @@ int bmgd_run_rounds_noalloc(const void* dev_x, const void* dev_y, int64_t rows, 
         rc = make_row_map(dev_x, rows, p, tb, var->cap(), &xmap);
         if (rc != BMGD_OK) return rc;
     }
-    cudaError_t e = cudaLaunchKernelEx(&lc, var->fn(L.threads + 32 * L.pwarps), P, xmap);
+    cudaError_t e = cudaLaunchKernelEx(&lc, var->fn(L.threads + 32 * L.pwarps, bmgdk::glm_flavour(P.opt_kind, P.sched, L.cpc)), P, xmap);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return (e == cudaErrorCooperativeLaunchTooLarge || e == cudaErrorLaunchOutOfResources) ? BMGD_ERR_LAUNCH : BMGD_ERR_CUDA;
@@ -1116,13 +1085,33 @@ const char* bmgd_strerror(int status) {
 int bmgd_last_cuda_error(const bmgd_t* h) { return h ? h->last_cuda : 0; }
 
 #ifdef BMGD_TRACE
+}  // extern "C"
+namespace bmgdk {
+// Debug build only: the two stamp arrays, allocated and zeroed on the device that is current at the first call (the
+// trace reader works on one device).  Null if that fails: the kernels then take no stamps.
+long long* trace_buffer(int which) {
+    static long long* buf[2] = {nullptr, nullptr};
+    static std::once_flag once;
+    std::call_once(once, [] {
+        const size_t bytes = sizeof(long long) * (size_t)kTraceBlocks * kTraceSteps * kTracePhases;
+        for (int i = 0; i < 2; ++i) {
+            void* ptr = nullptr;
+            if (cudaMalloc(&ptr, bytes) != cudaSuccess || cudaMemset(ptr, 0, bytes) != cudaSuccess) { cudaGetLastError(); ptr = nullptr; }
+            buf[i] = static_cast<long long*>(ptr);
+        }
+    });
+    return (which == 0 || which == 1) ? buf[which] : nullptr;
+}
+}  // namespace bmgdk
+extern "C" {
 // Debug build only: copy out the clock stamps [block][step][phase] that thread 0 of every CTA took at the phase
 // boundaries of its first steps (which = 0), or those of every CTA's first producer warp (which = 1).
 int bmgd_debug_trace(int which, long long* out_host, int count) {
     const int total = bmgdk::kTraceBlocks * bmgdk::kTraceSteps * bmgdk::kTracePhases;
     if (!out_host || count <= 0 || count > total || which < 0 || which > 1) return BMGD_ERR_ARG;
-    cudaError_t e = which == 0 ? cudaMemcpyFromSymbol(out_host, bmgdk::g_trace, sizeof(long long) * (size_t)count)
-                               : cudaMemcpyFromSymbol(out_host, bmgdk::g_ptrace, sizeof(long long) * (size_t)count);
+    const long long* src = bmgdk::trace_buffer(which);
+    if (!src) return BMGD_ERR_CUDA;
+    cudaError_t e = cudaMemcpy(out_host, src, sizeof(long long) * (size_t)count, cudaMemcpyDeviceToHost);
     return e == cudaSuccess ? BMGD_OK : BMGD_ERR_CUDA;
 }
 int bmgd_debug_trace_dims(int* blocks, int* steps, int* phases) {

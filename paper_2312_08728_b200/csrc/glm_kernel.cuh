@@ -46,6 +46,7 @@ constexpr unsigned long long kDrainNs = 1000000ull;  // at the end of a launch: 
 constexpr int kCtaAbortOff = 512;  // shared-memory word (in front of the ring) through which a CTA's consumers agree to stop
 constexpr int kOptSgd = 0, kOptNesterov = 1, kOptAdam = 2;  // == BMGD_OPT_*
 constexpr int kLrConstant = 0, kLrCosine = 1;               // == BMGD_LR_*
+constexpr int kGlmAny = 0, kGlmPlainOne = 1, kGlmPlainTeam = 2, kGlmFlavours = 3;  // see glm_kernel
 
 struct GlmParams {
     const void* X;        // [N0][p] rows
@@ -87,6 +88,10 @@ struct GlmParams {
     uint32_t chain0;      // shuffle id of this launch's first chain (chains of one job may be spread over several handles)
     uint32_t poll_mask;   // a packet poll looks at the clock and the abort flag every poll_mask+1 failed sweeps
     uint32_t mbar_mask;   // the same for the waits on the ring's mbarriers
+#ifdef BMGD_TRACE
+    long long* trace;     // debug build: clock stamps of thread 0 of every CTA, [block][step][phase] (null: none taken)
+    long long* ptrace;    // and of the first producer warp, per pair of ring stages
+#endif
 };
 
 // ---------------------------------------------------------------- small PTX wrappers
@@ -270,18 +275,18 @@ __host__ __device__ inline GlmSmemPlan glm_smem_plan(int warps, int gpw, bool pr
 // Debug build only (build.py, trace=True): clock stamps of thread 0 of every CTA at the phase boundaries of its first
 // steps, and of the first producer warp per pair of ring stages: the SM's cycle counter.
 constexpr int kTraceBlocks = 64, kTraceSteps = 48, kTracePhases = 16;
-__device__ long long g_trace[kTraceBlocks * kTraceSteps * kTracePhases];
-__device__ long long g_ptrace[kTraceBlocks * kTraceSteps * kTracePhases];
+long long* trace_buffer(int which);  // host: the device array of the consumers' (0) or producers' (1) stamps, zeroed when first asked for
+// The stamps go to two arrays of kTraceBlocks * kTraceSteps * kTracePhases words that the host hands over in the
+// kernel's parameters (P.trace, P.ptrace; null: no stamps).
 #define BMGD_STAMP(ph)                                                                                        \
     do {                                                                                                      \
-        if (threadIdx.x == 0 && blockIdx.x < (unsigned)kTraceBlocks && step_count < (uint32_t)kTraceSteps) {    \
-            g_trace[((int)blockIdx.x * kTraceSteps + (int)step_count) * kTracePhases + (ph)] = clock64();     \
-        }                                                                                                     \
+        if (threadIdx.x == 0 && P.trace && blockIdx.x < (unsigned)kTraceBlocks && step_count < (uint32_t)kTraceSteps) \
+            P.trace[((int)blockIdx.x * kTraceSteps + (int)step_count) * kTracePhases + (ph)] = clock64();     \
     } while (0)
 #define BMGD_PSTAMP(ph)                                                                                       \
     do {                                                                                                      \
-        if (pw == 0 && lane == 0 && blockIdx.x < (unsigned)kTraceBlocks && (it >> 1) < (uint32_t)kTraceSteps)   \
-            g_ptrace[((int)blockIdx.x * kTraceSteps + (int)(it >> 1)) * kTracePhases + (ph)] = clock64();     \
+        if (pw == 0 && lane == 0 && P.ptrace && blockIdx.x < (unsigned)kTraceBlocks && (it >> 1) < (uint32_t)kTraceSteps) \
+            P.ptrace[((int)blockIdx.x * kTraceSteps + (int)(it >> 1)) * kTracePhases + (ph)] = clock64();     \
     } while (0)
 #else
 #define BMGD_STAMP(ph) do { } while (0)
@@ -542,7 +547,14 @@ __device__ __forceinline__ void bounded_mbar_wait(uint32_t bar, uint32_t parity,
 // NULLSTEP = true is the latency probe of the same kernel: every wait, barrier, packet exchange and update of a step
 // runs with the same launch shape, but no row is fetched and none is multiplied (the gradient is zero and theta
 // stays as it is).  Its time per step is what the step's synchronisation structure alone costs.
-template <typename T, int VEC, int LPR, int KCH, bool LOGISTIC, int MAXT, bool NULLSTEP = false>
+//
+// FLAVOUR says which of the step's options a compiled kernel carries.  The step from one theta to the next is a chain
+// of dependent phases a few thousand cycles long, so the code of options that a launch does not use (the exchange
+// between clusters, the update rules with state, the rate schedule) costs time on that chain even when it is only
+// branched around: measured on B200, 10 to 14 % of the step of a chain that runs inside one cluster.  kGlmAny decides
+// everything at run time; the two plain flavours are Eq. (2.1) with a constant rate, compiled for a chain inside one
+// cluster (kGlmPlainOne) or spread over several (kGlmPlainTeam).  All flavours do the same arithmetic in the same order.
+template <typename T, int VEC, int LPR, int KCH, bool LOGISTIC, int MAXT, int FLAVOUR = kGlmAny, bool NULLSTEP = false>
 __global__ void __launch_bounds__(MAXT, 1)
 glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
     constexpr int GPW = 32 / LPR;            // row groups per warp
@@ -563,7 +575,11 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
     const int W = P.consumer_warps, NPW = P.producer_warps;  // blockDim.x == 32 * (W + NPW)
     const int nthreads = W * 32;                             // consumer threads: the ones that reduce and exchange
     const int warp = tid >> 5, lane = tid & 31;
-    const int S = P.S, cpc = P.cpc, G = cpc * S;
+    constexpr bool PLAIN = FLAVOUR != kGlmAny;
+    const int S = P.S, cpc = (FLAVOUR == kGlmPlainOne) ? 1 : P.cpc, G = cpc * S;
+    const bool one_cluster = (FLAVOUR == kGlmPlainOne) ? true : (FLAVOUR == kGlmPlainTeam) ? false : cpc == 1;
+    const int opt_kind = PLAIN ? kOptSgd : P.opt_kind;
+    const bool cosine = !PLAIN && P.sched == kLrCosine;
     const int rank = (S > 1) ? (int)cluster_ctarank() : 0;
     const int cluster_id = blockIdx.x / S;
     const int team = cluster_id / cpc, kc = cluster_id % cpc;
@@ -573,7 +589,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
     const int T_rounds = P.T, passes = P.passes, RB = P.rb, D = P.depth;
     const int spp = W * GPW;  // rows the CTA works on at once (one sub-pass)
 
-    const GlmSmemPlan plan = glm_smem_plan(W, GPW, PRE, RB, D, PCAP, (int)sizeof(T), S, cpc > 1, G4);
+    const GlmSmemPlan plan = glm_smem_plan(W, GPW, PRE, RB, D, PCAP, (int)sizeof(T), S, !one_cluster, G4);
     const int pitch = plan.pitch;
     const int stage_bytes = plan.stage_bytes;
     const uint32_t full_bars = smem_u32(smem), empty_bars = smem_u32(smem) + 128u;  // one 8-byte mbarrier per stage each
@@ -819,14 +835,14 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
         int fw_log2 = 5;  // predictors rounded up to a power of two of at least a warp
         while ((1 << fw_log2) < p) ++fw_log2;
         // threads that share a predictor's pushes: a power of two, at most S (cluster sizes are powers of two)
-        const int xg_n = (FPT == 1 && cpc == 1 && S > 1) ? max(1, min(S, nthreads >> fw_log2)) : 1;
+        const int xg_n = (FPT == 1 && one_cluster && S > 1) ? max(1, min(S, nthreads >> fw_log2)) : 1;
         const int xf = (xg_n > 1) ? (tid & ((1 << fw_log2) - 1)) : tid, xg = (xg_n > 1) ? (tid >> fw_log2) : 0;
         // Where this thread's packets go in its peers' shared memory (parity 0; the other parity lies a fixed distance
         // behind), worked out once when a thread has at most four peers to serve: the address arithmetic and the mapping
         // into the peer's window would otherwise be redone in every step, on the path from one theta to the next.
         constexpr int kFastPeers = 4;
         const int my_peers = (S + xg_n - 1 - xg) / xg_n;  // peers xg, xg + xg_n, ... below S
-        const bool fast_push = FPT == 1 && cpc == 1 && S > 1 && S / xg_n <= kFastPeers;
+        const bool fast_push = FPT == 1 && one_cluster && S > 1 && S / xg_n <= kFastPeers;
         uint32_t push_addr[kFastPeers];
 #pragma unroll
         for (int i = 0; i < kFastPeers; ++i)
@@ -863,8 +879,8 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
             for (int i = 0; i < FPT; ++i) {
                 const int f = tid + i * nthreads;
                 thm[i] = (f < p) ? theta_g[f] : T(0);
-                st1[i] = (f < p && P.opt_kind != kOptSgd) ? st1_g[f] : T(0);
-                st2[i] = (f < p && P.opt_kind == kOptAdam) ? st2_g[f] : T(0);
+                st1[i] = (f < p && opt_kind != kOptSgd) ? st1_g[f] : T(0);
+                st2[i] = (f < p && opt_kind == kOptAdam) ? st2_g[f] : T(0);
             }
             double b1pow = P.adam_b1pow0, b2pow = P.adam_b2pow0;  // beta^t after the steps of earlier calls
             long long sched_pos = P.sched_pos0;                   // updates already taken in this pass
@@ -949,7 +965,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                     const uint32_t tag = P.tag_base + step_count + 1u;
                     const uint32_t cpk = cpk_base + (uint32_t)(parity * S * plan.cpk_stride * 8);
 
-                    if (cpc == 1) {
+                    if (one_cluster) {
                         // ---- one cluster per chain: every CTA pushes its partial sums, as tagged packets, into the
                         //      shared memory of every CTA of the cluster and then sums, in rank order, the S packets per
                         //      predictor that arrive in its own.  No cluster barrier: a packet is its own flag.
@@ -1069,19 +1085,19 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                     //      then every lane refreshes the coefficients it multiplies rows with
                     const bool full = full_batch;
                     T lr = lr_const;
-                    if (P.sched == kLrCosine) {  // Section 4.4: rate of the j-th update of a pass of J updates
+                    if (cosine) {  // Section 4.4: rate of the j-th update of a pass of J updates
                         const long long j = sched_pos + 1;
                         lr = (T)(P.lr * (0.5 + 0.5 * cospi((double)j / (double)P.sched_period)));
                         sched_pos = (j == P.sched_period) ? 0 : j;
                     }
-                    if (P.opt_kind == kOptSgd) {
-                        const T scale = (P.sched == kLrCosine) ? lr * (full ? inv_full : inv_last) : (full ? scale_full : scale_last);
+                    if (opt_kind == kOptSgd) {
+                        const T scale = cosine ? lr * (full ? inv_full : inv_last) : (full ? scale_full : scale_last);
 #pragma unroll
                         for (int i = 0; i < FPT; ++i) {
                             const int f = tid + i * nthreads;
                             if (f < p) { thm[i] = fma(-scale, tot[i], thm[i]); gfin[f] = thm[i]; }
                         }
-                    } else if (P.opt_kind == kOptNesterov) {
+                    } else if (opt_kind == kOptNesterov) {
                         const T inv = full ? inv_full : inv_last, mu = (T)P.opt_a;
 #pragma unroll
                         for (int i = 0; i < FPT; ++i) {
@@ -1138,8 +1154,8 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                     const int f = tid + i * nthreads;
                     if (f < p) {
                         theta_g[f] = thm[i];
-                        if (P.opt_kind != kOptSgd) st1_g[f] = st1[i];
-                        if (P.opt_kind == kOptAdam) st2_g[f] = st2[i];
+                        if (opt_kind != kOptSgd) st1_g[f] = st1[i];
+                        if (opt_kind == kOptAdam) st2_g[f] = st2[i];
                     }
                 }
             }
@@ -1151,35 +1167,6 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
         cluster_arrive_release();
         cluster_wait_acquire();
     }
-}
-
-// Waits, with the step kernel's protocol, for a packet tag that nobody writes: the wait must run out of its
-// budget, record BMGD_ERR_TIMEOUT in the status word, raise the abort flag and return.  For testing the error path.
-__global__ void wait_probe_kernel(const unsigned long long* packet, uint32_t tag, unsigned long long timeout_ns, int* status) {
-    unsigned long long t0 = 0;
-    uint32_t spins = 0;
-    bool aborted = false;
-    while (!aborted) {
-        if ((uint32_t)(ld_packet(packet) >> 32) == tag) break;
-        if ((++spins & 0x3FFu) == 0u) {
-            const unsigned long long now = global_ns();
-            if (t0 == 0) t0 = now;
-            if (now - t0 > timeout_ns || ((volatile int*)status)[1] != 0) {
-                atomicCAS(status, 0, kStatusTimeout);
-                atomicExch(status + 1, 1);
-                aborted = true;
-            }
-        }
-    }
-}
-
-// Writes out[j] = pi(j) for one (seed, chain, round): the shuffle exactly as the step kernel uses it.
-__global__ void perm_kernel(unsigned long long seed, uint32_t chain, uint32_t round, uint32_t N0, uint32_t* out) {
-    const FeistelDomain dom = make_domain(N0);
-    const RoundKeys rk = round_keys(seed, chain, round);
-    for (unsigned long long j = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x; j < N0;
-         j += (unsigned long long)gridDim.x * blockDim.x)
-        out[j] = perm_index((uint32_t)j, dom, rk);
 }
 
 }  // namespace bmgdk

@@ -1,0 +1,5 @@
+#include "glm_table.cuh"
+
+namespace bmgdk {
+const GlmVariant* glm_variants_f32_linear(bool aligned16, int* count) { return glm_variants<float, false, false>(aligned16, count); }
+}  // namespace bmgdk

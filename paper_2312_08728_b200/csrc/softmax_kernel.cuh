@@ -63,6 +63,9 @@ struct SoftmaxParams {
     uint32_t chain0;
     int fixed_partition;
     uint32_t mbar_mask;
+#ifdef BMGD_TRACE
+    long long* trace;   // debug build: clock stamps of thread 0 of every CTA (null: none taken)
+#endif
 };
 
 struct SoftmaxLaunchInfo {
@@ -688,6 +691,9 @@ inline int softmax_run(const void* dx, const void* dy, int64_t rows, int p, int 
     const bool tiny = timeout_ns < 1000ull;  // below a microsecond: no budget at all, every failed look gives up
     if (tiny) P.timeout_ns = 0;
     P.mbar_mask = tiny ? 0u : 0x3Fu;
+#ifdef BMGD_TRACE
+    P.trace = trace_buffer(0);
+#endif
 
     e = cudaLaunchKernelEx(&lc, fn, P);
     if (e != cudaSuccess) { info->cuda_error = (int)e; cudaGetLastError(); return e == cudaErrorLaunchOutOfResources ? -7 : -3; }
