@@ -924,7 +924,11 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                         if (nsub) row_step<T, VEC, LPR, KCH, LOGISTIC>(rowp, yp, th, gacc);
                         if (sidx == 0) BMGD_STAMP(13);
                         __syncwarp();  // every lane has its values in registers: the slot may be refilled
-                        if (lane == 0) mbar_arrive(empty_bars + (uint32_t)(cs_slot * 8));
+                        // A lane that has given up did not wait for the stage and must not hand its slot back: a producer
+                        // would refill it while copies of the phase before are in flight, the phases of the slot's barrier
+                        // would run into one another, and the wait for the last copies at the end of the launch would
+                        // no longer mean that they have landed.
+                        if (lane == 0 && !aborted) mbar_arrive(empty_bars + (uint32_t)(cs_slot * 8));
                         if (++cs_slot == D) { cs_slot = 0; cs_phase ^= 1u; }
                     }
                     BMGD_STAMP(1);

@@ -46,6 +46,7 @@ constexpr int kSmxClasses = 16;      // padded class count
 // in registers after the read-out).  Measured on B200: a 128 x 16 x 16 multiply-accumulate takes about 70 cycles of the
 // tensor core whether or not it accumulates into the tile of the one before it, so more than one accumulator only adds
 // read-outs (four of them: forward 2,590 -> 2,730 cycles, backward 1,940 -> 2,250).
+constexpr unsigned long long kSmxLingerNs = 20000ull;  // how long a CTA of a launch that was given up stays before it exits
 constexpr int kSmxAcc = 1;
 constexpr int kSmxTmemCols = 4 * kSmxAcc * kSmxClasses;  // forward halves 0 and 1, backward tiles 0 and 1
 
@@ -621,6 +622,13 @@ __global__ void __launch_bounds__(kSmxThreads, 1) softmax_kernel(const SoftmaxPa
         __syncwarp();
         cluster_arrive_release();
         cluster_wait_acquire();
+        // In a launch that was given up, pieces sent with st.async may count on barriers that nobody waits for any more,
+        // and nothing else says when they have landed.  Every peer has stopped sending by now (the barrier above), and a
+        // piece is under way for well below a microsecond: the CTA stays for twenty before it gives up its shared memory.
+        if (reinterpret_cast<volatile int*>(P.status)[1] != 0) {
+            const unsigned long long t0 = global_ns();
+            while (global_ns() - t0 < kSmxLingerNs) { }
+        }
     }
 }
 
