@@ -88,7 +88,9 @@ typedef struct bmgd_config {
     int32_t threads_per_cta;  /* linear/logistic: threads that compute, a multiple of 32 from 256 to 512 (softmax: fixed) */
     int32_t pipeline_depth;   /* row-prefetch stages held in shared memory: 2 to 8 */
     int32_t subpasses_per_stage; /* a stage holds this many sweeps of the CTA over its rows: 1, 2, 4, ... 32 */
-    int32_t producer_warps;   /* linear/logistic: extra warps per CTA that only evaluate the shuffle and fetch rows: 1 to 8 */
+    int32_t producer_warps;   /* linear/logistic: extra warps per CTA that only evaluate the shuffle and fetch rows: 1 to 8
+                                 (rows that are not fetched by four-row gathers, i.e. not 16-byte multiples or wider than 256
+                                 values, get a multiple of pipeline_depth of them: the value is rounded to one) */
     int32_t lanes_per_row;    /* linear/logistic: lanes that share one row in the inner loop: 4, 8, 16 or 32, if the row size has
                                  a kernel built that way */
     int32_t first_chain;      /* shuffle id of this handle's first chain: chain c of the handle draws the partitions of

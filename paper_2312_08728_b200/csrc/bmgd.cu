@@ -270,11 +270,11 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     // gather).  Variants with wide per-lane state always run 8 consumer warps at 168 registers.
     const bool throughput = c.Rc > 1 && var->max_consumer_threads() >= 512;
     L.threads = c.threads_per_cta ? std::min(c.threads_per_cta, var->max_consumer_threads()) : (throughput ? 512 : 256);
-    // Producer warps only evaluate the shuffle and issue copies; both are chains of dependent instructions, so several
-    // warps side by side are what keeps them ahead of the consumers.
-    L.pwarps = c.producer_warps ? c.producer_warps : 4;
-    L.pwarps = std::min(L.pwarps, (var->max_threads() - L.threads) / 32);
-    if (L.pwarps < 1) return BMGD_ERR_ARG;
+    // Producer warps only evaluate the shuffle and issue copies; this is how many the CTA has room for.  Their number is
+    // settled below, once the ring is known: rows fetched by gathers are dealt to all producers stage by stage (4 by
+    // default), other layouts give every ring slot its own producer warp (or several that share its rows).
+    const int max_pwarps = std::min(8, (var->max_threads() - L.threads) / 32);
+    if (max_pwarps < 2) return BMGD_ERR_ARG;
     const int warps = L.threads / 32;
     const int spp = warps * gpw;  // rows a CTA works on at once (one sub-pass)
     const bool pre = bmgdk::glm_prereduce(var->kch * var->vec, var->lpr);
@@ -305,16 +305,21 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
             return BMGD_ERR_UNIMPLEMENTED;
         }
         const int probe_smem = fixed_smem + ring_budget;
-        // whichever flavour the launch takes in the end (that depends on the clusters per chain chosen below), it runs
-        // with these limits; all flavours have the same launch bounds, so one answers for all on residency
+        // whichever flavour and CTA size the launch takes in the end (they depend on the clusters per chain and the ring
+        // depth chosen below), it runs with these limits; a CTA takes nearly all of an SM's shared memory, so one
+        // instance answers for all on residency
         for (int fl = 0; fl < bmgdk::kGlmFlavours; ++fl) {
-            const void* fn = (const void*)var->fn(L.threads + 32 * L.pwarps, fl);
-            BMGD_CUDA(h, cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, probe_smem));
-            BMGD_CUDA(h, cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, S > 8 ? 1 : 0));
+            for (int size = 0; size < 2; ++size) {
+                const void* fn = (const void*)var->k[fl][size];
+                if (!fn) continue;
+                BMGD_CUDA(h, cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, probe_smem));
+                BMGD_CUDA(h, cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, S > 8 ? 1 : 0));
+            }
         }
         max_clusters = h->sm_count;
         if (S > 1) {
-            int rc = max_active_clusters(h, var->fn(L.threads + 32 * L.pwarps, bmgdk::kGlmAny), S, L.threads + 32 * L.pwarps, probe_smem, &max_clusters);
+            const int probe_threads = L.threads + 32 * max_pwarps;
+            int rc = max_active_clusters(h, var->fn(probe_threads, bmgdk::kGlmAny), S, probe_threads, probe_smem, &max_clusters);
             if (rc != BMGD_OK) {
                 if (c.cluster_size == 0 && S > 8) { S = 8; continue; }  // clusters of 16 are optional in hardware
                 return rc;
@@ -358,9 +363,13 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     // narrow rows (at most 32 bytes per lane) are swept four sub-passes at a time by the kernel, others two
     int rb = c.subpasses_per_stage ? c.subpasses_per_stage : ((var->kch * 16 <= 32) ? 4 : 2);
     rb = floor_pow2(std::max(1, std::min(rb, subpasses)));
-    // a producer warp takes at most kMaxBatchesPerProducer batches of 32 row slots per stage
-    while (rb > 1 && rb * spp > 32 * bmgdk::kMaxBatchesPerProducer * L.pwarps) rb /= 2;
-    if (spp > 32 * bmgdk::kMaxBatchesPerProducer * L.pwarps) return BMGD_ERR_ARG;
+    int shared_pwarps = 0;  // gathered rows: producer warps, all of which work on every stage
+    if (gathered) {
+        shared_pwarps = std::min(c.producer_warps ? c.producer_warps : 4, max_pwarps);
+        // a producer warp takes at most kMaxBatchesPerProducer batches of 32 row slots per stage
+        while (rb > 1 && rb * spp > 32 * bmgdk::kMaxBatchesPerProducer * shared_pwarps) rb /= 2;
+        if (spp > 32 * bmgdk::kMaxBatchesPerProducer * shared_pwarps) return BMGD_ERR_ARG;
+    }
     while (rb > 1 && 2 * stage_bytes_of(rb) > ring_budget) rb /= 2;
     L.rb = rb;
     L.passes = (subpasses + rb - 1) / rb;
@@ -368,9 +377,16 @@ int plan_glm(bmgd* h, const GlmVariant* var, int64_t rows, int n, LaunchShape* o
     // ring stages: 2 to 8.  Where partial sums cross clusters through global memory, copies in flight for later steps
     // delay the packets on the same path (measured on B200: cfg3 4.8 us per step with two stages, 5.7 with three).
     int depth = c.pipeline_depth ? c.pipeline_depth : (L.cpc > 1 ? 2 : 4);
+    if (!gathered) depth = std::min(depth, max_pwarps);  // one producer warp per ring slot at least
     while (depth > 2 && depth * stage_bytes > ring_budget) --depth;
     if (depth * stage_bytes > ring_budget) return BMGD_ERR_UNIMPLEMENTED;
     L.depth = depth;
+    if (gathered) {
+        L.pwarps = shared_pwarps;
+    } else {  // a multiple of the ring depth (cfg.producer_warps is rounded down to one; default: one per slot)
+        const int per_slot = std::max(1, std::min(c.producer_warps ? c.producer_warps : depth, max_pwarps) / depth);
+        L.pwarps = per_slot * depth;
+    }
     L.smem = bmgdk::glm_smem_plan(warps, gpw, pre, rb, depth, pcap, eb, S, multi, gathered).total_bytes;
     (void)rows;
     *out = L;

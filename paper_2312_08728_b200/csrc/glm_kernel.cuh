@@ -40,7 +40,7 @@ namespace bmgdk {
 
 constexpr int kMaxCpc = 20;        // clusters per chain the packet exchange is unrolled for
 constexpr int kMaxClusterSize = 16; // CTAs per cluster
-constexpr int kMaxBatchesPerProducer = 2;  // batches of 32 row slots one producer warp takes in one ring stage
+constexpr int kMaxBatchesPerProducer = 2;  // gathered rows: batches of 32 row slots one producer warp takes in one ring stage
 constexpr int kStatusTimeout = -5; // == BMGD_ERR_TIMEOUT
 constexpr unsigned long long kDrainNs = 1000000ull;  // at the end of a launch: how long a warp waits for its own copies in flight
 constexpr int kCtaAbortOff = 512;  // shared-memory word (in front of the ring) through which a CTA's consumers agree to stop
@@ -90,7 +90,7 @@ struct GlmParams {
     uint32_t mbar_mask;   // the same for the waits on the ring's mbarriers
 #ifdef BMGD_TRACE
     long long* trace;     // debug build: clock stamps of thread 0 of every CTA, [block][step][phase] (null: none taken)
-    long long* ptrace;    // and of the first producer warp, per pair of ring stages
+    long long* ptrace;    // and of the first producer warp, per pair of stages or per stage of its slot
 #endif
 };
 
@@ -273,7 +273,7 @@ __host__ __device__ inline GlmSmemPlan glm_smem_plan(int warps, int gpw, bool pr
 
 #ifdef BMGD_TRACE
 // Debug build only (build.py, trace=True): clock stamps of thread 0 of every CTA at the phase boundaries of its first
-// steps, and of the first producer warp per pair of ring stages: the SM's cycle counter.
+// steps, and of the first producer warp per pair of stages (gathered rows) or per stage of its slot: the SM's cycle counter.
 constexpr int kTraceBlocks = 64, kTraceSteps = 48, kTracePhases = 16;
 long long* trace_buffer(int which);  // host: the device array of the consumers' (0) or producers' (1) stamps, zeroed when first asked for
 // The stamps go to two arrays of kTraceBlocks * kTraceSteps * kTracePhases words that the host hands over in the
@@ -285,8 +285,8 @@ long long* trace_buffer(int which);  // host: the device array of the consumers'
     } while (0)
 #define BMGD_PSTAMP(ph)                                                                                       \
     do {                                                                                                      \
-        if (pw == 0 && lane == 0 && P.ptrace && blockIdx.x < (unsigned)kTraceBlocks && (it >> 1) < (uint32_t)kTraceSteps) \
-            P.ptrace[((int)blockIdx.x * kTraceSteps + (int)(it >> 1)) * kTracePhases + (ph)] = clock64();     \
+        if (pw == 0 && lane == 0 && P.ptrace && blockIdx.x < (unsigned)kTraceBlocks && pstep < (uint32_t)kTraceSteps) \
+            P.ptrace[((int)blockIdx.x * kTraceSteps + (int)pstep) * kTracePhases + (ph)] = clock64();         \
     } while (0)
 #else
 #define BMGD_STAMP(ph) do { } while (0)
@@ -302,12 +302,14 @@ __host__ __device__ constexpr int glm_max_consumer_threads() {
     return (sizeof(T) == 8 || KCH * VEC >= 24) ? 256 : 512;
 }
 // CTA sizes a kernel is compiled for (consumers plus producers; registers come in units of four warps): kGlmSmallCta
-// leaves 168 registers per thread, kGlmLargeCta 96 and is built only for variants with little per-lane state.  (A
-// 512-thread instance with 128 registers was measured too: never the fastest.)
-constexpr int kGlmSmallCta = 256 + 128, kGlmLargeCta = 512 + 128;
+// leaves 168 registers per thread, kGlmMidCta 128, kGlmLargeCta 96.  Every variant is built for the small size; fp32
+// variants also for a second one: with little per-lane state the large size (16 consumer warps), with wide per-lane
+// state the middle size, whose 8 consumer warps still fit 128 registers (a few bytes of spills) and which makes room
+// for 8 producer warps: replicate chains over wide rows are paced by their producers.
+constexpr int kGlmSmallCta = 256 + 128, kGlmMidCta = 256 + 256, kGlmLargeCta = 512 + 128;
 template <typename T, int VEC, int KCH>
 __host__ __device__ constexpr int glm_max_threads() {
-    return (sizeof(T) == 8 || KCH * VEC >= 24) ? kGlmSmallCta : kGlmLargeCta;
+    return sizeof(T) == 8 ? kGlmSmallCta : (KCH * VEC >= 24 ? kGlmMidCta : kGlmLargeCta);
 }
 // Fold the row groups of a warp together by shuffles before shared memory where that is cheap: few values per lane,
 // or only two groups per warp (one shuffle level).  Fewer partial rows also leave more shared memory for the ring.
@@ -345,9 +347,38 @@ __device__ __forceinline__ void perm_index2(uint32_t& x0, const RoundKeys& k0, u
             feistel_round_pair(L0, R0, k0.k[r], k0.k[r + 1], d);
             feistel_round_pair(L1, R1, k1.k[r], k1.k[r + 1], d);
         }
-        if (w0) { x0 = L0 * d.c + R0; w0 = x0 >= d.N0; }
-        if (w1) { x1 = L1 * d.c + R1; w1 = x1 >= d.N0; }
+        x0 = w0 ? L0 * d.c + R0 : x0;  // selects, not branches: the chains stay side by side
+        x1 = w1 ? L1 * d.c + R1 : x1;
+        w0 = w0 && x0 >= d.N0;
+        w1 = w1 && x1 >= d.N0;
     } while (w0 || w1);
+}
+
+// N indices of one round through the shuffle at once (the same round keys): the N Feistel chains are independent, so
+// their latencies overlap.
+template <int N>
+__device__ __forceinline__ void perm_index_n(uint32_t (&x)[N], const RoundKeys& rk, const FeistelDomain& d) {
+    bool walking[N];
+#pragma unroll
+    for (int i = 0; i < N; ++i) walking[i] = true;
+    bool any;
+    do {
+        uint32_t L[N], R[N];
+#pragma unroll
+        for (int i = 0; i < N; ++i) feistel_split(x[i], d, L[i], R[i]);
+#pragma unroll
+        for (int r = 0; r < 8; r += 2) {
+#pragma unroll
+            for (int i = 0; i < N; ++i) feistel_round_pair(L[i], R[i], rk.k[r], rk.k[r + 1], d);
+        }
+        any = false;
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+            x[i] = walking[i] ? L[i] * d.c + R[i] : x[i];  // selects, not branches: the chains stay side by side
+            walking[i] = walking[i] && x[i] >= d.N0;
+            any |= walking[i];
+        }
+    } while (any);
 }
 
 // The rare part of every bounded wait: look at the clock and at the launch's abort flag.  When the budget has run
@@ -603,7 +634,8 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
     if (tid < D) {
         // every producer lane, once its element copies have landed; with bulk row copies, also one lane per producer
         // warp announcing that warp's byte count
-        mbar_init(full_bars + (uint32_t)(tid * 8), (uint32_t)(NPW * (CB == 16 ? 33 : 32)));
+        // gathered rows: every producer warp; other layouts: the producer warps of this slot
+        mbar_init(full_bars + (uint32_t)(tid * 8), (uint32_t)((G4 ? NPW : NPW / D) * (CB == 16 ? 33 : 32)));
         mbar_init(empty_bars + (uint32_t)(tid * 8), (uint32_t)W);           // one lane of every consumer warp
     }
     fence_barrier_init();
@@ -619,13 +651,18 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
     if (warp >= W) {
         // ================================================================ producer warps
         // Rows do not depend on theta and the shuffle is stateless, so the producers run up to D stages ahead of
-        // the consumers, through mini-batch, round and chain boundaries.  Slots of a stage are taken 32 at a time
-        // (a batch; ownership of batches rotates over the producer warps): lane l evaluates pi for slot 32b + l and
-        // fetches that row, with one bulk copy when rows are 16-byte multiples.  Two consecutive stages are worked on
-        // together, so that their two shuffle evaluations overlap.
+        // the consumers, through mini-batch, round and chain boundaries.  Two schemes, by row layout (measured on B200):
+        //  * gathered rows (four rows per tensor-map gather): all producer warps work on the same stage, each on its
+        //    share of the stage's batches of 32 row slots, two consecutive stages together so that their shuffle
+        //    evaluations overlap.  The gathers of a stage are issued by several warps side by side, which is what the
+        //    copy engine wants (one warp issuing all 32 gathers of a stage: cfg2 4.06 instead of 3.69 us per step);
+        //  * other layouts (one bulk copy per row, or element-wise copies): producer warp pw serves ring slot pw % D
+        //    and nobody else's: it fills every stage that lands in that slot (stages slot, slot + D, ... of the launch)
+        //    independently of the other warps, so the shuffle evaluation for one slot overlaps the copies into the
+        //    others (p = 500, 100 chains: 24.0 instead of 27.2 us per step).  With NPW = nsub * D warps, the nsub
+        //    warps of a slot share a stage's batches.
         const int pw = warp - W;
-        const int R = RB * spp;
-        const int nbatch = (R + 31) >> 5;
+        const int R = RB * spp;  // row slots of a stage: a multiple of four
         const int nchunks = p / VEC;
         int lpr_c = 1;  // lanes that copy one row: the power of two at or above nchunks, at most 32
         while (lpr_c < nchunks && lpr_c < 32) lpr_c <<= 1;
@@ -638,7 +675,9 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
         const uint32_t row_bytes = (uint32_t)p * (uint32_t)sizeof(T);
         const FeistelDomain dom = make_domain(N0);
         const uint32_t ring_base = smem_u32(smem + plan.ring_off);
-
+        uint32_t issued_mask = 0, issued_par = 0;  // ring slots this warp has sent copies into, and the parity of the last such phase
+        if constexpr (G4) {
+        const int nbatch = (R + 31) >> 5;
         struct Cursor {  // which stage comes next, and what it needs
             int ci, t, sidx;
             uint32_t m;
@@ -665,11 +704,10 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
         uint32_t empty_parity = 1u;  // a fresh mbarrier lets a wait on parity 1 through
 
         // Copies the batch whose first slot is s0; lane l holds the row of slot s0 + l (kNoRow: the slot stays empty).
-        // Rows that are 16-byte multiples travel as one bulk copy each, counted in bytes on the stage's barrier (the
-        // return value is the number of rows this warp sent that way); others go element by element.
+        // Returns the number of gathers issued, whose bytes are counted on the stage's barrier.
         auto copy_batch = [&](uint32_t stage_base, uint32_t full_bar, int s0, uint32_t rows) -> uint32_t {
             const int left = R - s0;  // slots of this batch that exist
-            if constexpr (G4) {
+            {
                 // lane l < 8 fetches slots 4l..4l+3 with one gather; a slot without a row asks for the row behind the
                 // last one, which reads as zeros
                 const int q = (lane & 7) * 4;
@@ -686,54 +724,22 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                 }
                 // gathers issued for this batch: one per four slots that exist (the same in every lane: no vote needed)
                 return (uint32_t)min(8, (left + 3) >> 2);
-            } else if constexpr (CB == 16) {
-                const bool have = lane < left && rows != kNoRow;
-                const uint32_t dst = stage_base + (uint32_t)((s0 + lane) * pitch);
-                if (have) {
-                    bulk_copy_row(dst, Xrows + (size_t)rows * row_bytes, row_bytes, full_bar);
-                    cp_async_fill<(int)sizeof(T)>(dst + YOFF, yb + rows, true);
-                } else if (lane < left) {  // no row for this slot: it must contribute nothing
-                    for (int k = 0; k < nchunks; ++k) st_shared_zero16(dst + (uint32_t)(k * 16));
-                    st_shared_zero16(dst + YOFF);
-                    fence_async_proxy();  // a later bulk copy will overwrite these bytes
-                }
-                return (uint32_t)__popc(__ballot_sync(0xFFFFFFFFu, have));
-            } else {
-                const int iters = min(32, left + rpi - 1) / rpi;
-                for (int i = 0; i < iters; ++i) {
-                    const int sl = i * rpi + rsub;
-                    const uint32_t row = __shfl_sync(0xFFFFFFFFu, rows, sl);
-                    const bool have = row != kNoRow;
-                    const unsigned char* src = Xb + (have ? (size_t)row * row_bytes : 0);
-                    const uint32_t dst = stage_base + (uint32_t)((s0 + sl) * pitch + cl * CB);
-                    if (sl < left) {
-                        for (int k = 0; k < cpl; ++k) {
-                            const int ch = cl + k * lpr_c;
-                            if (ch < nchunks) cp_async_fill<CB>(dst + (uint32_t)(k * lpr_c * CB), src + (have ? (size_t)k * lpr_c * CB : 0), have);
-                        }
-                    }
-                }
-                if (lane < left) {
-                    const bool have = rows != kNoRow;
-                    cp_async_fill<(int)sizeof(T)>(stage_base + (uint32_t)((s0 + lane) * pitch + YOFF), yb + (have ? rows : 0u), have);
-                }
-                return 0u;
             }
         };
         // closes this warp's part of a stage: every lane arrives once its element copies have landed, one lane
         // announces the bytes of the warp's bulk copies
         auto finish_stage = [&](uint32_t full_bar, uint32_t bulk_rows) {  // bulk_rows: row copies, or gathers of four rows
             mbar_arrive_after_copies(full_bar);
-            if constexpr (CB == 16) {
-                __syncwarp();  // the zero fills of all lanes come before the announcing lane's arrival
-                if (lane == 0) mbar_arrive_expect_tx(full_bar, bulk_rows * (G4 ? (uint32_t)(4 * PCAP * (int)sizeof(T)) : row_bytes));
+            {
+                __syncwarp();
+                if (lane == 0) mbar_arrive_expect_tx(full_bar, bulk_rows * (uint32_t)(4 * PCAP * (int)sizeof(T)));
             }
         };
 
-        uint32_t issued_mask = 0, issued_par = 0;  // ring slots this warp has sent copies into, and the parity of the last such phase
         uint32_t rot = (uint32_t)pw;  // (pw - pair * nbatch) mod NPW, kept incrementally: ownership of batches rotates
         const uint32_t rot_step = (uint32_t)(nbatch % NPW);
         for (uint32_t it = 0; it < total_stages; it += 2) {
+            [[maybe_unused]] const uint32_t pstep = it >> 1;  // trace build: stamps per pair of stages
             BMGD_PSTAMP(0);
             const Cursor A = cur;
             advance(cur);
@@ -801,12 +807,141 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                 BMGD_PSTAMP(6);
             }
         }
+        } else {
+        const int slot = pw % D, sub = pw / D, nsub = NPW / D;  // the host launches a multiple of D producer warps
+        const uint32_t stage_base = ring_base + (uint32_t)(slot * stage_bytes);
+        const uint32_t full_bar = full_bars + (uint32_t)(slot * 8), empty_bar = empty_bars + (uint32_t)(slot * 8);
+
+        // Copies 32 consecutive row slots from s0 on; lane l holds the row of slot s0 + l (kNoRow: the slot stays empty).
+        // Layouts other than the gathered one: rows that are 16-byte multiples travel as one bulk copy each, counted in
+        // bytes on the stage's barrier (the return value is the number of rows sent that way); others go element by element.
+        auto copy_batch = [&](int s0, uint32_t rows) -> uint32_t {
+            const int left = R - s0;  // slots of this batch that exist
+            if constexpr (CB == 16) {
+                const bool have = lane < left && rows != kNoRow;
+                const uint32_t dst = stage_base + (uint32_t)((s0 + lane) * pitch);
+                if (have) {
+                    bulk_copy_row(dst, Xrows + (size_t)rows * row_bytes, row_bytes, full_bar);
+                    cp_async_fill<(int)sizeof(T)>(dst + YOFF, yb + rows, true);
+                } else if (lane < left) {  // no row for this slot: it must contribute nothing
+                    for (int k = 0; k < nchunks; ++k) st_shared_zero16(dst + (uint32_t)(k * 16));
+                    st_shared_zero16(dst + YOFF);
+                    fence_async_proxy();  // a later bulk copy will overwrite these bytes
+                }
+                return (uint32_t)__popc(__ballot_sync(0xFFFFFFFFu, have));
+            } else {
+                const int iters = min(32, left + rpi - 1) / rpi;
+                for (int i = 0; i < iters; ++i) {
+                    const int sl = i * rpi + rsub;
+                    const uint32_t row = __shfl_sync(0xFFFFFFFFu, rows, sl);
+                    const bool have = row != kNoRow;
+                    const unsigned char* src = Xb + (have ? (size_t)row * row_bytes : 0);
+                    const uint32_t dst = stage_base + (uint32_t)((s0 + sl) * pitch + cl * CB);
+                    if (sl < left) {
+                        for (int k = 0; k < cpl; ++k) {
+                            const int ch = cl + k * lpr_c;
+                            if (ch < nchunks) cp_async_fill<CB>(dst + (uint32_t)(k * lpr_c * CB), src + (have ? (size_t)k * lpr_c * CB : 0), have);
+                        }
+                    }
+                }
+                if (lane < left) {
+                    const bool have = rows != kNoRow;
+                    cp_async_fill<(int)sizeof(T)>(stage_base + (uint32_t)((s0 + lane) * pitch + YOFF), yb + (have ? rows : 0u), have);
+                }
+                return 0u;
+            }
+        };
+
+        // where the stage that this warp fills next sits in the job: chain of the team, round, mini-batch, ring stage of
+        // the step; kept by counting (D stages forward per stage filled)
+        int c_ci = 0, c_t = 0, c_sidx = 0;
+        uint32_t c_m = 0;
+        auto forward = [&](int stages) {
+            for (int i = 0; i < stages; ++i) {
+                if (++c_sidx == passes) {
+                    c_sidx = 0;
+                    if (++c_m == M) {
+                        c_m = 0;
+                        if (++c_t == T_rounds) { c_t = 0; ++c_ci; }
+                    }
+                }
+            }
+        };
+        forward(slot);
+        int k_ci = -1, k_t = -1;  // chain and round the keys below belong to
+        RoundKeys rk;
+        uint32_t empty_parity = 1u;  // a fresh mbarrier lets a wait on parity 1 through
+        constexpr int kPair = 2;     // batches of 32 row slots whose shuffle indices are evaluated side by side
+
+        for (uint32_t it = (uint32_t)slot; it < total_stages; it += (uint32_t)D) {
+            [[maybe_unused]] const uint32_t pstep = it / (uint32_t)D;  // trace build: stamps per stage of this warp's slot
+            BMGD_PSTAMP(0);
+            if (c_ci != k_ci || c_t != k_t) {
+                k_ci = c_ci; k_t = c_t;
+                rk = round_keys(P.seed, P.chain0 + (uint32_t)(team + c_ci * P.nteams), P.fixed_partition ? 0u : (uint32_t)c_t);
+            }
+            const RowShare sh = row_share(c_m, n, N0, (uint32_t)g, (uint32_t)G, P.q_full, P.r_full);
+            const uint32_t u0 = (uint32_t)(c_sidx * R);  // the stage's first row slot within this CTA's share of the mini-batch
+            uint32_t sent = 0;   // bulk row copies that this warp sends into the stage
+            bool waited = false;  // the slot is known to be empty
+            {
+                const int nbatch = (R + 31) >> 5;
+                for (int b0 = sub * kPair; b0 < nbatch; b0 += nsub * kPair) {
+                    uint32_t row[kPair];
+                    bool valid[kPair];
+#pragma unroll
+                    for (int j = 0; j < kPair; ++j) {
+                        const int s = 32 * (b0 + j) + lane;
+                        const uint32_t u = u0 + (uint32_t)s;
+                        valid[j] = !NULLSTEP && s < R && u < sh.cnt;
+                        row[j] = valid[j] ? sh.lo + sh.a + u : 0u;
+                    }
+                    if constexpr (!NULLSTEP) {
+                        if (__any_sync(0xFFFFFFFFu, valid[0] || valid[1])) perm_index_n<kPair>(row, rk, dom);
+                        __syncwarp();
+                    }
+                    if (!waited) {
+                        BMGD_PSTAMP(1);
+                        bounded_mbar_wait(empty_bar, empty_parity, aborted, P);
+                        aborted = __any_sync(0xFFFFFFFFu, aborted);
+                        if (aborted) break;  // the launch has been given up: no further copies are issued
+                        waited = true;
+                    }
+                    if constexpr (!NULLSTEP) {
+#pragma unroll
+                        for (int j = 0; j < kPair; ++j)
+                            if (b0 + j < nbatch) sent += copy_batch(32 * (b0 + j), valid[j] ? row[j] : kNoRow);
+                    }
+                }
+            }
+            if (aborted) break;
+            if (!waited) {  // a warp without a chunk in this stage still counts on its barrier
+                BMGD_PSTAMP(1);
+                bounded_mbar_wait(empty_bar, empty_parity, aborted, P);
+                aborted = __any_sync(0xFFFFFFFFu, aborted);
+                if (aborted) break;
+            }
+            BMGD_PSTAMP(3);
+            // closes this warp's part of the stage: every lane arrives once its element copies have landed, one lane
+            // announces the bytes of the warp's bulk copies
+            mbar_arrive_after_copies(full_bar);
+            if constexpr (CB == 16) {
+                __syncwarp();  // the zero fills of all lanes come before the announcing lane's arrival
+                if (lane == 0) mbar_arrive_expect_tx(full_bar, sent * row_bytes);
+            }
+            issued_mask = 1u << slot;
+            issued_par = (empty_parity ^ 1u) << slot;
+            empty_parity ^= 1u;
+            forward(D);
+            BMGD_PSTAMP(4);
+        }
+        }
         cp_async_wait_all();
         // No CTA may exit while bulk copies into its shared memory are in flight.  After a normal run the consumers
         // have waited for every stage; after a launch that was given up they have not, so every producer warp waits
         // here, for a bounded time, until the last phase it sent copies into has completed on each ring slot (a phase
-        // completes once all producers have arrived and all bytes have landed; if a producer gave up before arriving,
-        // the time limit ends the wait, long after the copies themselves have landed).
+        // completes once all producers of the slot have arrived and all bytes have landed; if one of them gave up before
+        // arriving, the time limit ends the wait, long after the copies themselves have landed).
         {
             const unsigned long long t0 = global_ns();
             for (int s = 0; s < D; ++s) {

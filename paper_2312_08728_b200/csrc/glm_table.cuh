@@ -11,7 +11,7 @@ namespace bmgdk {
 typedef void (*GlmKernel)(const GlmParams, const CUtensorMap);
 
 struct GlmVariant {
-    // [flavour][0: CTAs of up to kGlmSmallCta threads (more registers per thread), 1: up to kGlmLargeCta, or null]
+    // [flavour][0: CTAs of up to kGlmSmallCta threads (more registers per thread), 1: the variant's second size (glm_max_threads), or null]
     GlmKernel k[kGlmFlavours][2];
     GlmKernel fn(int cta_threads, int flavour) const {
         const int large = (cta_threads > kGlmSmallCta && k[flavour][1]) ? 1 : 0;

@@ -96,20 +96,24 @@ __host__ __device__ __forceinline__ uint32_t feistel_g(uint32_t v, uint32_t k, u
 // x -> (x div c, x mod c) for x < a c < 2^32.  mulhi(x, ceil(2^32 / c)) is the quotient or one more (the rounding up
 // of the reciprocal adds less than one to x / c); one more shows as a remainder that wrapped round.
 __host__ __device__ __forceinline__ void feistel_split(uint32_t x, const FeistelDomain& d, uint32_t& L, uint32_t& R) {
-    uint32_t q = mulhi32(x, d.inv_c);
-    uint32_t r = x - q * d.c;
-    if (r >= d.c) { q -= 1u; r += d.c; }
-    L = q;
-    R = r;
+    const uint32_t q = mulhi32(x, d.inv_c);
+    const uint32_t r = x - q * d.c;
+    const bool wrapped = r >= d.c;  // written as selects: a branch here would stand between the chains of several indices
+    L = wrapped ? q - 1u : q;
+    R = wrapped ? r + d.c : r;
+}
+
+// v mod m for v < 2 m, without a branch: v - m wraps round to a huge value exactly when v < m
+__host__ __device__ __forceinline__ uint32_t reduce_once(uint32_t v, uint32_t m) {
+    const uint32_t w = v - m;
+    return w < v ? w : v;
 }
 
 // two rounds of the network: both halves are below their moduli before and after
 __host__ __device__ __forceinline__ void feistel_round_pair(uint32_t& L, uint32_t& R, uint32_t k_even, uint32_t k_odd,
                                                             const FeistelDomain& d) {
-    L += feistel_g(R, k_even, d.a);
-    if (L >= d.a) L -= d.a;
-    R += feistel_g(L, k_odd, d.c);
-    if (R >= d.c) R -= d.c;
+    L = reduce_once(L + feistel_g(R, k_even, d.a), d.a);
+    R = reduce_once(R + feistel_g(L, k_odd, d.c), d.c);
 }
 
 __host__ __device__ __forceinline__ uint32_t perm_index(uint32_t j, const FeistelDomain& d, const RoundKeys& rk) {

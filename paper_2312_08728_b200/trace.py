@@ -52,7 +52,7 @@ PHASES_MULTI = [("step head", 0, 11), ("wait for 1st stage", 11, 10), ("1st stag
                 ("l2-poll+push", 12, 5), ("totals", 5, 6), ("update", 6, 9), ("reload", 9, 7)]
 PHASES_SOFTMAX = [("wait for rows", 0, 1), ("forward + read-out", 1, 2), ("logits exchange", 2, 3), ("softmax + R push", 3, 4),
                   ("R arrival", 4, 5), ("backward + read-out", 5, 6), ("update + barrier", 6, 7)]
-PRODUCER = [("shuffle", 0, 1), ("slot+copies A", 1, 3), ("arrive A", 3, 4), ("slot+copies+arrive B", 4, 6)]
+PRODUCER = [("shuffle", 0, 1), ("slot wait + copies (A)", 1, 3), ("arrive (A)", 3, 4), ("B (gathered rows)", 4, 6)]
 
 
 def trace_workload(L, spec):
@@ -106,7 +106,7 @@ def trace_workload(L, spec):
         d = np.median(pt[:nblk, steps, b] - pt[:nblk, steps, a], axis=1)
         print(f"   producer {label:22s} {int(d[0]):6d}   (CTAs: median {int(np.median(d)):6d})")
     pair = np.median(pt[:nblk, 9:t.shape[1] - 4, 0] - pt[:nblk, 8:t.shape[1] - 5, 0], axis=1)
-    print(f"   producer pair of stages: {int(pair[0])} cycles")
+    print(f"   producer warp 0, one turn of its loop (a pair of stages with gathered rows, else one stage of its slot): {int(pair[0])} cycles")
 
 
 def main(argv):
