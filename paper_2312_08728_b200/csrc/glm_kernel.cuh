@@ -994,6 +994,14 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
         int cs_slot = 0;         // ring slot the compute cursor reads next
         uint32_t cs_phase = 0;   // parity of that slot's "full" phase
         uint32_t step_count = 0; // steps this team has finished in this launch
+        // Where a step has an exchange to wait for, the wait for the next step's first ring stage is taken while this
+        // step's packets are under way (the stage has usually long been filled, but asking costs about 120 cycles, which
+        // would otherwise sit at the head of the next step, on the path from one theta to the next).
+        bool prewaited = false;
+        auto wait_next_stage_early = [&]() {
+            prewaited = (step_count + 1u) * (uint32_t)passes < total_stages;  // there is a next stage in this launch
+            if (prewaited) bounded_mbar_wait(full_bars + (uint32_t)(cs_slot * 8), cs_phase, aborted, P);
+        };
 
         for (int ci = 0; ci < nch; ++ci) {
             const int chain = team + ci * P.nteams;
@@ -1037,7 +1045,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                     if (!full_batch) sp_left = (sh.cnt > warp_first) ? (int)((sh.cnt - warp_first - 1u) / (uint32_t)spp) + 1 : 0;
                     for (int sidx = 0; sidx < passes; ++sidx) {
                         if (sidx == 0) BMGD_STAMP(11);
-                        bounded_mbar_wait(full_bars + (uint32_t)(cs_slot * 8), cs_phase, aborted, P);
+                        if (!(sidx == 0 && prewaited)) bounded_mbar_wait(full_bars + (uint32_t)(cs_slot * 8), cs_phase, aborted, P);
                         __syncwarp();
                         if (sidx == 0) BMGD_STAMP(10);
                         const unsigned char* rowp = smem + plan.ring_off + cs_slot * stage_bytes + lane_off;
@@ -1135,6 +1143,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                                 }
                             }
                             BMGD_STAMP(8);
+                            wait_next_stage_early();
     #pragma unroll
                             for (int i = 0; i < FPT; ++i) {
                                 const int f = tid + i * nthreads;
@@ -1165,6 +1174,7 @@ glm_kernel(const GlmParams P, const __grid_constant__ CUtensorMap xmap) {
                             }
                         }
                         BMGD_STAMP(4);
+                        wait_next_stage_early();
                         unsigned long long* slot = P.ll + ((size_t)(team * 2 + parity) * cpc) * (size_t)P.ll_stride;
                         const uint32_t gpk = gpk_base + (uint32_t)(parity * PCAP * NW * 8);
                         // thread j of the CTA owns predictor f = rank*slice + j of the slice (all of them if S == 1)
