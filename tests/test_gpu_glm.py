@@ -105,6 +105,22 @@ def test_producer_warps_ragged_batches_and_chains():
     check(w, buffers_of(w), mode="resident", producer_warps=1)
 
 
+@pytest.mark.parametrize("dtype,p", [(DTYPE_F32, 500), (DTYPE_F32, 33), (DTYPE_F64, 130), (DTYPE_F64, 7)])
+@pytest.mark.parametrize("shape", [
+    dict(cluster_size=1, ctas_per_chain=1),                                      # one producer warp per slot of the default ring
+    dict(cluster_size=1, ctas_per_chain=1, pipeline_depth=2, producer_warps=4),  # two warps share a slot's batches
+    dict(cluster_size=2, ctas_per_chain=4, pipeline_depth=3, producer_warps=1),  # rounded up to one warp per slot
+    dict(cluster_size=4, ctas_per_chain=4, pipeline_depth=2, subpasses_per_stage=1, producer_warps=3),
+    dict(cluster_size=2, ctas_per_chain=2, pipeline_depth=4, subpasses_per_stage=4),
+])
+def test_rows_not_fetched_by_gathers_have_one_producer_warp_per_ring_slot(dtype, p, shape):
+    """Rows wider than 256 values (one bulk copy per row) and rows that are not 16-byte multiples (element-wise copies)
+    are fetched by producer warps that each serve one ring slot; ring depths, warps per slot, chains that take turns on
+    a team and a ragged last mini-batch must all give the oracle's theta."""
+    w = Workload("slots", LOSS_LOGISTIC, dtype, N=2_300, p=p, K=1, n=300, T=2, lr=0.3, epochs=1, Rc=3, seed=200 + p)
+    check(w, buffers_of(w), mode="resident", **shape)
+
+
 def test_cluster_of_sixteen_if_the_device_allows_it():
     from paper_2312_08728_b200.binding import BmgdError
     try:
