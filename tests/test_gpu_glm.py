@@ -112,6 +112,8 @@ def test_producer_warps_ragged_batches_and_chains():
     dict(cluster_size=2, ctas_per_chain=4, pipeline_depth=3, producer_warps=1),  # rounded up to one warp per slot
     dict(cluster_size=4, ctas_per_chain=4, pipeline_depth=2, subpasses_per_stage=1, producer_warps=3),
     dict(cluster_size=2, ctas_per_chain=2, pipeline_depth=4, subpasses_per_stage=4),
+    dict(cluster_size=1, ctas_per_chain=2, pipeline_depth=8, subpasses_per_stage=1),  # more slots than the small CTA has warps for
+    dict(cluster_size=2, ctas_per_chain=2, pipeline_depth=6, subpasses_per_stage=1, producer_warps=8),
 ])
 def test_rows_not_fetched_by_gathers_have_one_producer_warp_per_ring_slot(dtype, p, shape):
     """Rows wider than 256 values (one bulk copy per row) and rows that are not 16-byte multiples (element-wise copies)
