@@ -86,7 +86,8 @@ typedef struct bmgd_config {
     int32_t cluster_size;     /* CTAs per thread-block cluster: 1, 2, 4, 8 or 16 */
     int32_t ctas_per_chain;
     int32_t threads_per_cta;  /* linear/logistic: threads that compute, a multiple of 32 from 256 to 512 (softmax: fixed) */
-    int32_t pipeline_depth;   /* row-prefetch stages held in shared memory: 2 to 8 */
+    int32_t pipeline_depth;   /* row-prefetch stages held in shared memory: 2 to 8 (fewer where shared memory, or the
+                                 warps a CTA has room for, do not allow as many: bmgd_get_stats reports what ran) */
     int32_t subpasses_per_stage; /* a stage holds this many sweeps of the CTA over its rows: 1, 2, 4, ... 32 */
     int32_t producer_warps;   /* linear/logistic: extra warps per CTA that only evaluate the shuffle and fetch rows: 1 to 8
                                  (rows that are not fetched by four-row gathers, i.e. not 16-byte multiples or wider than 256
